@@ -1,0 +1,55 @@
+"""The composed entry points of the path, built from the single steps.
+
+Test infrastructure (see the package header).
+
+w4a4_linear : per-token scale + static quantise -> INT4 matmul -> scale factors
+              (Sec. 3.1.3; App. B "Static quantization"; App. J "Setup")
+decoder_mlp : one SwiGLU MLP block in the normalised-residual form of Sec. 3.1.3
+              X~_n = RMSNorm(Z~_{n-1}),  S_n = S_{n-1} / ||Z~_{n-1}||_R   (Eq. 7)
+              g, u = W4A4 linears of X~_n
+              m    = bf16(silu(g) * u), quantised after the multiply by S_n
+                     (the scaler placed at the down-projection input)
+              Y~_n = W4A4 down projection of S_n * m  (= S_n * Y_n, Eq. 5)
+              Z~_n = X~_n + Y~_n   when the residual is requested
+"""
+import numpy as np
+
+from .quantizers import QParams, act_quant, silu_mul_quant
+from .int_matmul import int_matmul
+from .epilogue import dequant_epilogue, inverse_of_pre
+
+F32 = np.float32
+
+POST_NONE = 0
+POST_INVERSE_OF_PRE = 1
+POST_VECTOR = 2
+
+
+def w4a4_linear(x, wq, sw, qp, rmsnorm=True, scale_input=False, eps=1e-5, s_in=None,
+                post_mode=POST_NONE, post=None):
+    """Returns dict(codes, acc, y, s_out, p)."""
+    codes, s_out, p, r = act_quant(x, qp, rmsnorm, scale_input, eps, s_in)
+    acc = int_matmul(codes, wq, qp.z)
+    if post_mode == POST_NONE:
+        pv = None
+    elif post_mode == POST_INVERSE_OF_PRE:
+        pv = inverse_of_pre(p)
+    else:
+        pv = np.asarray(post, dtype=F32)
+    y = dequant_epilogue(acc, sw, qp.scale, pv)
+    return dict(codes=codes, acc=acc, y=y, s_out=s_out, p=p, r=r)
+
+
+def decoder_mlp(x, wg_q, sw_g, wu_q, sw_u, wd_q, sw_d, qp_in, qp_mid, eps=1e-5,
+                s_prev=None, add_residual=False):
+    """Returns dict(xq, g, u, m, mq, y, s_out)."""
+    xq, s_n, p, r = act_quant(x, qp_in, rmsnorm=True, scale_input=False, eps=eps, s_in=s_prev)
+    g = dequant_epilogue(int_matmul(xq, wg_q, qp_in.z), sw_g, qp_in.scale)
+    u = dequant_epilogue(int_matmul(xq, wu_q, qp_in.z), sw_u, qp_in.scale)
+    mq, m = silu_mul_quant(g, u, qp_mid, s_n)
+    acc_d = int_matmul(mq, wd_q, qp_mid.z)
+    res = None
+    if add_residual:
+        res = (np.asarray(x, dtype=F32) * r[:, None]).astype(F32)     # X~_n = Z~_{n-1} / rho
+    y = dequant_epilogue(acc_d, sw_d, qp_mid.scale, None, res)
+    return dict(xq=xq, g=g, u=u, m=m, mq=mq, acc_d=acc_d, y=y, s_out=s_n, r=r)
