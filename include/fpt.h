@@ -1,0 +1,216 @@
+/*
+ * fpt.h -- C ABI of the B200 (sm_100a) statically quantised W4A4 linear path.
+ *
+ * The path is the transformer linear layer that FPTQuant makes viable with static
+ * INT4 activations: once the mergeable transforms are folded into the weights
+ * (Sec. 3.1.1, 3.1.2), every projection is
+ *   (1) RMSNorm-derived per-token scale + static INT4 quantise + pack   (Sec. 3.1.3, App. B)
+ *   (2) packed-INT4 x packed-INT4 matmul with an exact INT32 accumulator (App. J)
+ *   (3) floating-point scale factors applied after the integer matmul   (App. B)
+ *
+ * General rules
+ *   - Every pointer is a DEVICE pointer unless it is a `const fpt_qparams*` (HOST).
+ *   - The caller owns every buffer.  The library allocates no device memory and keeps
+ *     no state between calls except a per-process cache of driver entry points.
+ *   - `stream` is a cudaStream_t passed as void*.  Work is enqueued on it and the call
+ *     returns without synchronising, except fpt_check_status.
+ *   - Row-major, contiguous tensors.  Activations are X[M, K] (one row per token);
+ *     weights are stored W[N, K] = [out features, in features], so Y = X W^T.
+ *   - Packed INT4: byte j of a row holds code 2j in bits 0..3 and code 2j+1 in bits
+ *     4..7 ("double-packed", App. J); symmetric grids store two's complement nibbles,
+ *     asymmetric grids store unsigned nibbles.
+ *   - Pointers to packed tensors, bf16 tensors and workspaces are 16-byte aligned;
+ *     K is a multiple of 32 (fpt_act_quant, fpt_quantize_weights) and of 128 for the
+ *     matmul entry points; N is a multiple of 8.
+ *   - Every function returns FPT_OK (0) or a negative error code; nothing throws,
+ *     aborts or traps.  Argument errors are detected before anything is enqueued.
+ *   - Floating point is float32 with one rounding per operation (no fused
+ *     multiply-add on the quantisation path); bf16 narrowing is round-to-nearest-even.
+ *
+ * Quantiser grid (the paper states "uniform integer grid", Sec. 1, with scale and
+ * offset as parameters, App. D; the formula is this library's reading):
+ *   symmetric : q = clamp(rne(v / D), -2^(b-1), 2^(b-1)-1)        v^ = D q
+ *   asymmetric: q = clamp(rne(v / D) + z, 0, 2^b - 1)             v^ = D (q - z)
+ * rne = round to nearest, ties to even.  v / D is evaluated as v * (1/D) with 1/D
+ * rounded once to float32 on the host.  A NaN maps to the lowest code.
+ */
+#ifndef FPT_H_
+#define FPT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- error codes -------------------------------------------------------------- */
+#define FPT_OK                0
+#define FPT_ERR_BAD_ARG      -1   /* null pointer, non-positive size, bad enum          */
+#define FPT_ERR_UNSUPPORTED  -2   /* bits != 4, K or N not a supported multiple, ...    */
+#define FPT_ERR_ALIGNMENT    -3   /* a pointer or leading dimension is misaligned       */
+#define FPT_ERR_WORKSPACE    -4   /* workspace missing or smaller than required         */
+#define FPT_ERR_CUDA         -5   /* a CUDA runtime / driver call failed                */
+#define FPT_ERR_TIMEOUT      -6   /* a device-side wait gave up (see fpt_check_status)  */
+
+/* ---- enums -------------------------------------------------------------------- */
+#define FPT_DTYPE_BF16 0
+#define FPT_DTYPE_F32  1
+#define FPT_DTYPE_F16  2
+
+#define FPT_RANGE_MINMAX 0        /* L_inf range setting: D = max|w| / qmax             */
+#define FPT_RANGE_LP     1        /* L_p range setting (App. D): least sum |w - w^|^p   */
+
+/* flags of fpt_act_quant / fpt_w4a4_linear */
+#define FPT_RMSNORM         1     /* r_t = 1/sqrt(mean_k x^2 + eps); the grid sees x * r_t        */
+#define FPT_SCALE_INPUT     2     /* the grid sees x * s_in[t] (times r_t when FPT_RMSNORM too)   */
+#define FPT_SILU_MUL        4     /* x := bf16(silu(X) * X2) before anything else (no RMSNORM)    */
+#define FPT_GU_INTERLEAVED  8     /* with FPT_SILU_MUL: X holds gate||up in 128-column groups     */
+
+/* where the per-token scale ends up after the matmul (Sec. 3.1.3: the scale commutes
+ * with a bias-free linear, so the caller chooses) */
+#define FPT_POST_NONE            0   /* y = (acc * sw[n]) * D_a                                   */
+#define FPT_POST_INVERSE_OF_PRE  1   /* ... * (D_a * (1 / p_t)), p_t the multiplier used in (1)   */
+#define FPT_POST_VECTOR          2   /* ... * (D_a * post[t])                                     */
+
+#define FPT_OP_LINEAR 0
+#define FPT_OP_MLP    1
+#define FPT_OP_GEMM   2
+
+/* One quantiser, as the paper parametrises it: bit-width, grid kind, static scale and
+ * offset (App. D "General set-up"). HOST struct. */
+typedef struct fpt_qparams {
+  int   bits;        /* 4 */
+  int   symmetric;   /* 1: codes in [-8, 7], zero_point ignored; 0: codes in [0, 15]     */
+  float scale;       /* static per-tensor scale D (activations); ignored for weights,    */
+                     /* whose per-output-channel scales are computed                     */
+  int   zero_point;  /* z of the asymmetric grid                                          */
+} fpt_qparams;
+
+int         fpt_version(void);
+const char* fpt_strerror(int code);
+
+/*
+ * Offline weight quantiser (uniform grid, round-to-nearest, per-output-channel scale;
+ * Sec. 4 "Quantization Setup", App. D "Quantizer range setting").
+ *   W        [N, K] device, bf16 or f32 (w_dtype)
+ *   qp       host; bits = 4, symmetric = 1 (weights always use the symmetric grid)
+ *   range    FPT_RANGE_MINMAX: D_n = max_k|w_nk| / 7
+ *            FPT_RANGE_LP    : D_n = (a_n * (i/100)) / 7 for the i in 20..100 with the least
+ *                              sum_k |w - D clamp(rne(w/D))|^p (float64), ties to larger i
+ *   scale_dtype  FPT_DTYPE_F32 or FPT_DTYPE_F16: D_n is rounded to it BEFORE the codes
+ *            are computed; an all-zero row gets D_n = 1
+ *   Wq       [N, K/2] out, packed codes q = clamp(rne(w / D_n), -8, 7) (IEEE division)
+ *   sw       [N] out, scale_dtype
+ *   wsum     [N] out int32, sum_k q_nk; may be NULL (needed only for asymmetric activations)
+ */
+int fpt_quantize_weights(void* stream, const void* W, int w_dtype, int N, int K,
+                         const fpt_qparams* qp, int range_mode, float p, int scale_dtype,
+                         uint8_t* Wq, void* sw, int32_t* wsum);
+
+/*
+ * Copies separately quantised gate and up matrices into the row-interleaved layout that
+ * fpt_decoder_mlp expects: for every group r of 128 output features, rows
+ * [256 r, 256 r + 128) of Wgu_q are gate rows [128 r, 128 r + 128) and rows
+ * [256 r + 128, 256 r + 256) are the matching up rows; sw_gu follows the same order.
+ * d_ff must be a multiple of 128.  (No counterpart in the paper: it is a storage choice
+ * that lets one matmul tile hold a gate column and its up column.)
+ */
+int fpt_interleave_gate_up(void* stream, const uint8_t* Wg_q, const uint8_t* Wu_q,
+                           const void* sw_g, const void* sw_u, int scale_dtype,
+                           int d_ff, int K, uint8_t* Wgu_q, void* sw_gu);
+
+/*
+ * Step (1): per-token scale + static quantise + pack (Sec. 3.1.3 Eq. 6-7; App. B).
+ * Per token t (row of X):
+ *   x_tk  = X[t,k]                                   (FPT_SILU_MUL: bf16(silu(X[t,k]) * X2[t,k]))
+ *   r_t   = 1 / sqrt( (float)(sum_k x_tk^2 in float64) / K + eps )      if FPT_RMSNORM else 1
+ *   p_t   = r_t * s_in[t]   if FPT_SCALE_INPUT (s_in required)          else r_t
+ *   q_tk  = clamp(rne((x_tk * p_t) * (1/D)) + z)
+ *   s_out[t] = r_t * s_in[t] if s_in != NULL else r_t      -- S_n = S_{n-1} / ||Z~_{n-1}||_R
+ * A block input uses FPT_RMSNORM alone (the grid sees RMSNorm(x), s_out carries the
+ * recursion); a site inside a block (attention output, down-projection input) uses
+ * FPT_SCALE_INPUT alone (the grid sees S_n x).
+ *   X      [M, ldx] bf16, ldx >= K elements, ldx % 8 == 0
+ *   X2     second operand of FPT_SILU_MUL, same layout as X; with FPT_GU_INTERLEAVED X2 is
+ *          ignored, X is [M, 2K] (ldx >= 2K) and logical column k lives at
+ *          gate: (k/128)*256 + k%128, up: gate + 128
+ *   s_in   [M] f32 or NULL;  s_out [M] f32 or NULL
+ *   Xq     [M, K/2] packed codes out
+ * silu(g) = g / (1 + 2^(-g*log2 e)) with a fixed float32 polynomial for 2^f (degree 6
+ * Taylor, Horner, separately rounded multiply and add), so that the result is one
+ * defined float32 value.
+ */
+int fpt_act_quant(void* stream, const void* X, int M, int K, int ldx,
+                  const fpt_qparams* qp, int flags, float eps,
+                  const void* X2, const float* s_in, uint8_t* Xq, float* s_out);
+
+/*
+ * Steps (2)+(3) on already packed operands (App. J "Setup"; App. B "Static quantization"):
+ *   acc[t,n] = sum_k (qa[t,k] - z) * qw[n,k]                 exact int32
+ *   y[t,n]   = bf16( ((float)acc * sw[n]) * c_t  [+ res[t,n] * res_scale[t]] )
+ *   c_t      = act_scale * post[t]  (post != NULL)  else act_scale
+ *   Xq [M, K/2], Wq [N, K/2] packed; sw [N] (scale_dtype); wsum [N] int32, required
+ *   when act_symmetric == 0; post [M] f32 or NULL.
+ *   residual [M, N] bf16 or NULL, added in float32 before the single bf16 rounding;
+ *   res_scale [M] f32 or NULL (1).
+ *   Y [M, N] bf16 out (may be NULL when acc_out is given)
+ *   acc_out [M, N] int32 or NULL: debugging aid, the raw accumulators.
+ *   workspace: fpt_workspace_bytes(FPT_OP_GEMM, M, N, K) bytes; its first word is the
+ *   status word read by fpt_check_status.
+ * M >= 1; K % 128 == 0; N % 8 == 0.  For M <= 64 a weight-streaming kernel is used.
+ */
+int fpt_w4a4_gemm(void* stream, const uint8_t* Xq, const uint8_t* Wq, int M, int N, int K,
+                  const void* sw, int scale_dtype, const int32_t* wsum,
+                  float act_scale, int act_symmetric, int act_zero_point,
+                  const float* post, const void* residual, const float* res_scale,
+                  void* Y, int32_t* acc_out, void* workspace, size_t workspace_bytes);
+
+/*
+ * Steps (1)+(2)+(3): one W4A4 linear on bf16 activations.
+ *   X [M, K] bf16; flags / eps / s_in / s_out as in fpt_act_quant (FPT_SILU_MUL not allowed);
+ *   post_mode selects c_t (see FPT_POST_*); post [M] only for FPT_POST_VECTOR.
+ *   workspace: fpt_workspace_bytes(FPT_OP_LINEAR, M, N, K) bytes (packed activations,
+ *   the per-token vectors and the status word live there).
+ */
+int fpt_w4a4_linear(void* stream, const void* X, int M, int K,
+                    const uint8_t* Wq, const void* sw, int scale_dtype, const int32_t* wsum, int N,
+                    const fpt_qparams* act_qp, int flags, float eps, const float* s_in,
+                    int post_mode, const float* post,
+                    void* Y, float* s_out, void* workspace, size_t workspace_bytes);
+
+/*
+ * One SwiGLU MLP block in the normalised-residual form of Sec. 3.1.3:
+ *   X~ = RMSNorm(X),  S_n = S_{n-1} * r                       (X is Z~_{n-1}; Eq. 7)
+ *   g, u = W4A4 linears of X~ (bf16)                          grid qp_in
+ *   m = bf16(silu(g) * u);  quantise m * S_n                  grid qp_mid (scaler at the
+ *                                                              down-projection input)
+ *   Y~ = W4A4 down projection  (= S_n * Y_n, Eq. 5)
+ *   Y  = bf16(Y~ + X * r)  if add_residual  (Z~_n = X~_n + Y~_n)   else bf16(Y~)
+ *   Wgu_q [2 d_ff, d/2] and sw_gu [2 d_ff] in the layout of fpt_interleave_gate_up;
+ *   Wd_q [d, d_ff/2], sw_d [d]; s_prev [M] or NULL (= 1); s_out [M] or NULL.
+ *   d % 128 == 0, d_ff % 128 == 0.  Both grids symmetric in this version.
+ *   workspace: fpt_workspace_bytes(FPT_OP_MLP, M, d_ff, d) bytes.
+ */
+int fpt_decoder_mlp(void* stream, const void* X, int M, int d, int d_ff,
+                    const uint8_t* Wgu_q, const void* sw_gu, const uint8_t* Wd_q, const void* sw_d,
+                    int scale_dtype, const fpt_qparams* qp_in, const fpt_qparams* qp_mid, float eps,
+                    const float* s_prev, float* s_out, int add_residual,
+                    void* Y, void* workspace, size_t workspace_bytes);
+
+/* Bytes of caller-provided scratch an entry point needs (op = FPT_OP_*).
+ * FPT_OP_LINEAR / FPT_OP_GEMM: (M, N, K); FPT_OP_MLP: (M, d_ff, d). */
+size_t fpt_workspace_bytes(int op, int M, int N, int K);
+
+/* Zeroes the status word of a workspace (call once after allocating it). */
+int fpt_reset_status(void* stream, void* workspace);
+
+/* Synchronises `stream`, reads the status word at the start of `workspace` and returns
+ * FPT_OK, FPT_ERR_TIMEOUT (a bounded device-side wait expired; the kernel released its
+ * resources and returned, outputs are invalid) or FPT_ERR_CUDA. */
+int fpt_check_status(void* stream, void* workspace);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FPT_H_ */

@@ -64,10 +64,10 @@ class QParams:
 # grid primitives
 # --------------------------------------------------------------------------- #
 def round_clamp(u, z, qmin, qmax):
-    """codes = clamp(rne(u) + z, qmin, qmax); a NaN maps to clamp(z)."""
+    """codes = clamp(rne(u) + z, qmin, qmax); a NaN maps to the lowest code."""
     u = np.asarray(u, dtype=F32)
     v = np.rint(u) + F32(z)                      # rint: ties to even
-    v = np.where(np.isnan(v), F32(min(max(z, qmin), qmax)), v)
+    v = np.where(np.isnan(v), F32(qmin), v)
     v = np.minimum(np.maximum(v, F32(qmin)), F32(qmax))
     return v.astype(np.int8 if qmin < 0 else np.uint8)
 

@@ -1,0 +1,170 @@
+// C-ABI entry points that compose the kernels: argument checks, workspace carving,
+// launches.  No device memory is allocated here; everything lives in caller buffers.
+#include "fpt_internal.cuh"
+
+namespace fpt {
+
+static inline size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+static int check_qp(const fpt_qparams* qp) {
+  if (!qp) return FPT_ERR_BAD_ARG;
+  if (qp->bits != 4) return FPT_ERR_UNSUPPORTED;
+  if (!(qp->scale > 0.0f)) return FPT_ERR_BAD_ARG;
+  if (!qp->symmetric && (qp->zero_point < 0 || qp->zero_point > 15)) return FPT_ERR_BAD_ARG;
+  return FPT_OK;
+}
+
+static int check_gemm_shape(int M, int N, int K) {
+  if (M <= 0 || N <= 0 || K <= 0) return FPT_ERR_BAD_ARG;
+  if (K % 128 != 0 || K > 65535 || N % 8 != 0) return FPT_ERR_UNSUPPORTED;
+  return FPT_OK;
+}
+
+}  // namespace fpt
+
+using namespace fpt;
+
+extern "C" int fpt_version(void) { return 100; }
+
+extern "C" const char* fpt_strerror(int code) {
+  switch (code) {
+    case FPT_OK: return "ok";
+    case FPT_ERR_BAD_ARG: return "bad argument";
+    case FPT_ERR_UNSUPPORTED: return "unsupported size, bit-width or combination of flags";
+    case FPT_ERR_ALIGNMENT: return "misaligned pointer or leading dimension";
+    case FPT_ERR_WORKSPACE: return "workspace missing or too small";
+    case FPT_ERR_CUDA: return "CUDA call failed";
+    case FPT_ERR_TIMEOUT: return "a device-side wait gave up";
+    default: return "unknown error code";
+  }
+}
+
+extern "C" size_t fpt_workspace_bytes(int op, int M, int N, int K) {
+  if (M <= 0 || N <= 0 || K <= 0) return 0;
+  const size_t m = (size_t)M;
+  switch (op) {
+    case FPT_OP_GEMM:
+      return kStatusBytes;
+    case FPT_OP_LINEAR:
+      return kStatusBytes + up256(m * (size_t)K / 2) + up256(m * 4);
+    case FPT_OP_MLP: {   // N = d_ff, K = d
+      const size_t dff = (size_t)N, d = (size_t)K;
+      return kStatusBytes + up256(m * d / 2) + 2 * up256(m * 4) + up256(m * 2 * dff * 2) + up256(m * dff / 2);
+    }
+    default:
+      return 0;
+  }
+}
+
+extern "C" int fpt_reset_status(void* stream, void* workspace) {
+  if (!workspace) return FPT_ERR_BAD_ARG;
+  return cudaMemsetAsync(workspace, 0, kStatusBytes, (cudaStream_t)stream) == cudaSuccess ? FPT_OK : FPT_ERR_CUDA;
+}
+
+extern "C" int fpt_check_status(void* stream, void* workspace) {
+  if (!workspace) return FPT_ERR_BAD_ARG;
+  uint32_t word = 0;
+  if (cudaMemcpyAsync(&word, workspace, 4, cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess)
+    return FPT_ERR_CUDA;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return FPT_ERR_CUDA;
+  return word == 0 ? FPT_OK : FPT_ERR_TIMEOUT;
+}
+
+extern "C" int fpt_w4a4_gemm(void* stream, const uint8_t* Xq, const uint8_t* Wq, int M, int N, int K, const void* sw,
+                             int scale_dtype, const int32_t* wsum, float act_scale, int act_symmetric,
+                             int act_zero_point, const float* post, const void* residual, const float* res_scale,
+                             void* Y, int32_t* acc_out, void* workspace, size_t workspace_bytes) {
+  if (!Xq || !Wq || !sw || (!Y && !acc_out)) return FPT_ERR_BAD_ARG;
+  int rc = check_gemm_shape(M, N, K);
+  if (rc) return rc;
+  if (scale_dtype != FPT_DTYPE_F32 && scale_dtype != FPT_DTYPE_F16) return FPT_ERR_BAD_ARG;
+  if (!(act_scale > 0.0f)) return FPT_ERR_BAD_ARG;
+  if (!act_symmetric && (!wsum || act_zero_point < 0 || act_zero_point > 15)) return FPT_ERR_BAD_ARG;
+  if (((uintptr_t)Xq | (uintptr_t)Wq | (uintptr_t)Y | (uintptr_t)acc_out | (uintptr_t)residual | (uintptr_t)workspace) & 15)
+    return FPT_ERR_ALIGNMENT;
+  if (!workspace || workspace_bytes < fpt_workspace_bytes(FPT_OP_GEMM, M, N, K)) return FPT_ERR_WORKSPACE;
+  GemmParams P{};
+  P.M = M; P.N = N; P.K = K;
+  P.sw = sw; P.scale_dtype = scale_dtype;
+  P.wsum = act_symmetric ? nullptr : wsum;
+  P.zero_point = act_symmetric ? 0 : act_zero_point;
+  P.a_unsigned = act_symmetric ? 0 : 1;
+  P.act_scale = act_scale;
+  P.post = post;
+  P.residual = reinterpret_cast<const __nv_bfloat16*>(residual);
+  P.res_scale = res_scale;
+  P.Y = reinterpret_cast<__nv_bfloat16*>(Y);
+  P.acc_out = acc_out;
+  P.status = reinterpret_cast<uint32_t*>(workspace);
+  return gemm_launch((cudaStream_t)stream, Xq, Wq, P);
+}
+
+extern "C" int fpt_w4a4_linear(void* stream, const void* X, int M, int K, const uint8_t* Wq, const void* sw,
+                               int scale_dtype, const int32_t* wsum, int N, const fpt_qparams* act_qp, int flags,
+                               float eps, const float* s_in, int post_mode, const float* post, void* Y, float* s_out,
+                               void* workspace, size_t workspace_bytes) {
+  if (!X || !Wq || !sw || !Y) return FPT_ERR_BAD_ARG;
+  int rc = check_qp(act_qp);
+  if (rc) return rc;
+  rc = check_gemm_shape(M, N, K);
+  if (rc) return rc;
+  if (flags & ~(FPT_RMSNORM | FPT_SCALE_INPUT)) return FPT_ERR_UNSUPPORTED;
+  if ((flags & FPT_SCALE_INPUT) && !s_in) return FPT_ERR_BAD_ARG;
+  if (post_mode < FPT_POST_NONE || post_mode > FPT_POST_VECTOR) return FPT_ERR_BAD_ARG;
+  if (post_mode == FPT_POST_VECTOR && !post) return FPT_ERR_BAD_ARG;
+  if (!act_qp->symmetric && !wsum) return FPT_ERR_BAD_ARG;
+  if (((uintptr_t)X | (uintptr_t)Wq | (uintptr_t)Y | (uintptr_t)workspace) & 15) return FPT_ERR_ALIGNMENT;
+  if (!workspace || workspace_bytes < fpt_workspace_bytes(FPT_OP_LINEAR, M, N, K)) return FPT_ERR_WORKSPACE;
+  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+  uint8_t* Xq = ws + kStatusBytes;
+  float* post_inv = reinterpret_cast<float*>(Xq + up256((size_t)M * K / 2));
+  cudaStream_t st = (cudaStream_t)stream;
+  if (act_quant_launch(st, X, M, K, K, act_qp, flags, eps, nullptr, s_in, Xq, s_out,
+                       post_mode == FPT_POST_INVERSE_OF_PRE ? post_inv : nullptr, nullptr) != cudaSuccess)
+    return FPT_ERR_CUDA;
+  const float* pv = post_mode == FPT_POST_NONE ? nullptr : post_mode == FPT_POST_VECTOR ? post : post_inv;
+  return fpt_w4a4_gemm(stream, Xq, Wq, M, N, K, sw, scale_dtype, wsum, act_qp->scale, act_qp->symmetric,
+                       act_qp->zero_point, pv, nullptr, nullptr, Y, nullptr, workspace, kStatusBytes);
+}
+
+extern "C" int fpt_decoder_mlp(void* stream, const void* X, int M, int d, int d_ff, const uint8_t* Wgu_q,
+                               const void* sw_gu, const uint8_t* Wd_q, const void* sw_d, int scale_dtype,
+                               const fpt_qparams* qp_in, const fpt_qparams* qp_mid, float eps, const float* s_prev,
+                               float* s_out, int add_residual, void* Y, void* workspace, size_t workspace_bytes) {
+  if (!X || !Wgu_q || !sw_gu || !Wd_q || !sw_d || !Y) return FPT_ERR_BAD_ARG;
+  int rc = check_qp(qp_in);
+  if (rc) return rc;
+  rc = check_qp(qp_mid);
+  if (rc) return rc;
+  if (!qp_in->symmetric || !qp_mid->symmetric) return FPT_ERR_UNSUPPORTED;
+  if (M <= 0 || d <= 0 || d_ff <= 0) return FPT_ERR_BAD_ARG;
+  if (d % 128 != 0 || d_ff % 128 != 0 || d_ff > 32768 || d > 65535) return FPT_ERR_UNSUPPORTED;
+  if (scale_dtype != FPT_DTYPE_F32 && scale_dtype != FPT_DTYPE_F16) return FPT_ERR_BAD_ARG;
+  if (((uintptr_t)X | (uintptr_t)Wgu_q | (uintptr_t)Wd_q | (uintptr_t)Y | (uintptr_t)workspace) & 15)
+    return FPT_ERR_ALIGNMENT;
+  if (!workspace || workspace_bytes < fpt_workspace_bytes(FPT_OP_MLP, M, d_ff, d)) return FPT_ERR_WORKSPACE;
+  const size_t m = (size_t)M;
+  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+  uint8_t* Xq = ws + kStatusBytes;
+  float* sn_ws = reinterpret_cast<float*>(Xq + up256(m * d / 2));
+  float* r_ws = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(sn_ws) + up256(m * 4));
+  uint8_t* GU = reinterpret_cast<uint8_t*>(r_ws) + up256(m * 4);
+  uint8_t* Mq = GU + up256(m * 2 * (size_t)d_ff * 2);
+  float* sn = s_out ? s_out : sn_ws;
+  cudaStream_t st = (cudaStream_t)stream;
+
+  // X~ = RMSNorm(X) on the grid qp_in; S_n = S_{n-1} * r
+  if (act_quant_launch(st, X, M, d, d, qp_in, FPT_RMSNORM, eps, nullptr, s_prev, Xq, sn, nullptr, r_ws) != cudaSuccess)
+    return FPT_ERR_CUDA;
+  // gate || up in one matmul over the interleaved weight
+  rc = fpt_w4a4_gemm(stream, Xq, Wgu_q, M, 2 * d_ff, d, sw_gu, scale_dtype, nullptr, qp_in->scale, 1, 0, nullptr,
+                     nullptr, nullptr, GU, nullptr, workspace, kStatusBytes);
+  if (rc) return rc;
+  // m = bf16(silu(g) * u), quantised after the multiply by S_n
+  if (act_quant_launch(st, GU, M, d_ff, 2 * d_ff, qp_mid, FPT_SILU_MUL | FPT_GU_INTERLEAVED | FPT_SCALE_INPUT, 0.0f,
+                       nullptr, sn, Mq, nullptr, nullptr, nullptr) != cudaSuccess)
+    return FPT_ERR_CUDA;
+  // down projection; the normalised residual X * r joins before the final rounding
+  return fpt_w4a4_gemm(stream, Mq, Wd_q, M, d, d_ff, sw_d, scale_dtype, nullptr, qp_mid->scale, 1, 0, nullptr,
+                       add_residual ? X : nullptr, add_residual ? r_ws : nullptr, Y, nullptr, workspace, kStatusBytes);
+}

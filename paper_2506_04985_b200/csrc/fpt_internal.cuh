@@ -1,0 +1,33 @@
+// Declarations shared between the translation units of the library (host side).
+#pragma once
+
+#include "fpt_common.cuh"
+
+namespace fpt {
+
+struct GemmParams {
+  int M, N, K;
+  int tiles_m, num_tiles, kblocks;
+  const void* sw;
+  int scale_dtype;
+  const int32_t* wsum;
+  int zero_point;              // 0 when the activation grid is symmetric
+  int a_unsigned;              // activation codes are unsigned nibbles (asymmetric grid)
+  float act_scale;
+  const float* post;
+  const __nv_bfloat16* residual;
+  const float* res_scale;
+  __nv_bfloat16* Y;
+  int32_t* acc_out;
+  uint32_t* status;
+};
+
+// act_quant.cu: validated arguments only; also fills 1/p_t and r_t for the composed calls.
+cudaError_t act_quant_launch(cudaStream_t st, const void* X, int M, int K, int ldx, const fpt_qparams* qp,
+                             int flags, float eps, const void* X2, const float* s_in, uint8_t* Xq,
+                             float* s_out, float* post_inv, float* r_out);
+
+// gemm_w4a4.cu: validated arguments only; returns an FPT_* code.
+int gemm_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, const GemmParams& P);
+
+}  // namespace fpt

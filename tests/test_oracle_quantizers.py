@@ -63,7 +63,7 @@ def test_round_ties_to_even_table():
     u = np.array([0.5, 1.5, 2.5, -0.5, -1.5, -2.5, 3.5, 6.5, 7.5, -8.5, 100.0, -100.0], dtype=F32)
     assert Q.round_clamp(u, 0, -8, 7).tolist() == [0, 2, 2, 0, -2, -2, 4, 6, 7, -8, 7, -8]
     assert Q.round_clamp(u, 8, 0, 15).tolist() == [8, 10, 10, 8, 6, 6, 12, 14, 15, 0, 15, 0]
-    assert Q.round_clamp(np.array([np.nan], dtype=F32), 0, -8, 7).tolist() == [0]
+    assert Q.round_clamp(np.array([np.nan], dtype=F32), 0, -8, 7).tolist() == [-8]
 
 
 @pytest.mark.parametrize("sym,z", [(True, 0), (False, 8), (False, 3)])
