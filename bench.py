@@ -1,0 +1,346 @@
+#!/usr/bin/env python
+"""Benchmark of the W4A4 static linear path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload attn|mlp]
+
+One step = one pass of the whole hot path over one batch of the Llama-3-8B-shaped
+attention projections at prefill (2048 tokens, hidden 4096): per-token scale + static INT4
+quantise of the block input, fused Q||K||V W4A4 matmul (N = 6144) with its scale-factor
+epilogue, then scale + quantise of the attention-output tensor and the O projection
+(N = 4096).  2*M*K*(6144+4096) = 171.8 GOP per step.  Inputs are seeded synthetic tensors
+(heavy-tailed activations with outlier channels, Gaussian weights, quantised offline).
+
+Prints ONE JSON line (rank 0): whole-job TOPS with inputs resident in HBM (`value`), the
+same through host buffers (`e2e`), the roofline of the dominant kernel measured live with
+CUDA events, clocks sampled during the timed region, and the CPU oracle timed on a bounded
+sample (`cpu_baseline`).  `--impl reference` times the oracle alone.
+"""
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+M_TOK, HID, N_QKV, N_O = 2048, 4096, 6144, 4096
+D_FF = 14336
+EPS = 1e-5
+NSETS = 4
+METRIC = "W4A4 linear TOPS (prefill, Llama-3-8B-shaped attention projections, 2048 tokens)"
+
+
+def step_ops(workload):
+    if workload == "mlp":
+        return 2.0 * 4096 * HID * D_FF * 3
+    return 2.0 * M_TOK * HID * (N_QKV + N_O)
+
+
+# ------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU through NVML (read-only) while alive."""
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.reasons, self.stop_flag = index, [], set(), False
+        self.max_mhz, self.ok = None, False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        while self.ok and not self.stop_flag:
+            try:
+                self.samples.append(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM))
+                r = self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                for bit, name in self.REASONS.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.05)
+
+    def result(self):
+        self.stop_flag = True
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["unavailable"]}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------------------------------
+# CPU oracle leg (cpu_baseline and --impl reference)
+# ------------------------------------------------------------------------------------------
+def oracle_sample_setup(rows):
+    from oracle import quantizers as OQ
+    from paper_2506_04985_b200 import synth
+    x = synth.f32(synth.activations(rows, HID, 0, "bench/x0", law="student_t3", outlier_frac=0.005, outlier_gain=50.0))
+    ao = synth.f32(synth.activations(rows, HID, 0, "bench/ao0", law="student_t3", outlier_frac=0.005,
+                                     outlier_gain=50.0))
+    s_in = synth.per_token_scale(rows, 0, "bench/s0").numpy()
+    wqkv = synth.f32(synth.weights(N_QKV, HID, 0.02, 0, "bench/wqkv0"))
+    wo = synth.f32(synth.weights(N_O, HID, 0.02, 0, "bench/wo0"))
+    cq, dq, _ = OQ.quantize_weights(wqkv)
+    co, do, _ = OQ.quantize_weights(wo)
+    return dict(x=x, ao=ao, s_in=s_in, cq=cq, dq=dq, co=co, do=do)
+
+
+def oracle_sample_step(S, qp_x, qp_o):
+    from oracle import linear as OL
+    a = OL.w4a4_linear(S["x"], S["cq"], S["dq"], qp_x, True, False, EPS)
+    b = OL.w4a4_linear(S["ao"], S["co"], S["do"], qp_o, False, True, EPS, S["s_in"])
+    return a["y"], b["y"]
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else os.cpu_count()
+    except Exception:
+        return os.cpu_count()
+
+
+def time_oracle(rows, reps):
+    from oracle.quantizers import QParams as OQP
+    S = oracle_sample_setup(rows)
+    qp_x, qp_o = OQP(4, True, 0.45), OQP(4, True, 2.0)
+    oracle_sample_step(S, qp_x, qp_o)
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        oracle_sample_step(S, qp_x, qp_o)
+    dt = (time.perf_counter() - t0) / reps
+    ops = 2.0 * rows * HID * (N_QKV + N_O)
+    return ops / dt / 1e12, dt
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    # size the per-step sample so that warmup + steps end within about two minutes
+    _, dt256 = time_oracle(256, 1)
+    budget = 120.0 / max(1, args.steps + args.warmup)
+    rows = int(max(16, min(M_TOK, 256 * budget / dt256))) // 16 * 16
+    S = oracle_sample_setup(rows)
+    from oracle.quantizers import QParams as OQP
+    qp_x, qp_o = OQP(4, True, 0.45), OQP(4, True, 2.0)
+    for _ in range(args.warmup):
+        oracle_sample_step(S, qp_x, qp_o)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_sample_step(S, qp_x, qp_o)
+    dt = (time.perf_counter() - t0) / max(1, args.steps)
+    tops = 2.0 * rows * HID * (N_QKV + N_O) / dt / 1e12
+    cores = blas_threads()
+    sample = f"{rows} of {M_TOK} token rows x all {N_QKV + N_O} output columns per step (numpy oracle, float64 BLAS matmul)"
+    line = {"impl": "reference", "metric": METRIC, "value": tops, "unit": "TOPS", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int4 x int4 -> int32 (oracle: exact in float64)",
+            "data": "synthetic", "config": {"workload": "configs[1]: Llama-3-8B-shaped attention projections, "
+                                            "2048 tokens, hidden 4096, fused QKV (6144) + O (4096)",
+                                            "sampled_rows": rows},
+            "cpu_baseline": {"value": tops, "unit": "TOPS", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": tops, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------
+# GPU leg
+# ------------------------------------------------------------------------------------------
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_burst": d["bf16_tflops"], "bf16_sustained": d["bf16_tflops_sustained"],
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2506_04985_b200 import binding as B, synth, build
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl")
+    build.build()
+    B.lib()
+    dev = torch.device("cuda", local)
+
+    # ---- seeded inputs: NSETS rotating sets so that every step reads HBM, not L2 ------------
+    sets = []
+    for i in range(NSETS):
+        tag = f"{i + NSETS * rank}"
+        x = synth.activations(M_TOK, HID, 0, "bench/x" + tag, law="student_t3", outlier_frac=0.005, outlier_gain=50.0)
+        ao = synth.activations(M_TOK, HID, 0, "bench/ao" + tag, law="student_t3", outlier_frac=0.005, outlier_gain=50.0)
+        s_in = synth.per_token_scale(M_TOK, 0, "bench/s" + tag)
+        wqkv = synth.weights(N_QKV, HID, 0.02, 0, "bench/wqkv" + tag).to(dev)
+        wo = synth.weights(N_O, HID, 0.02, 0, "bench/wo" + tag).to(dev)
+        wq1, sw1, _ = B.fpt_quantize_weights(wqkv)
+        wq2, sw2, _ = B.fpt_quantize_weights(wo)
+        del wqkv, wo
+        sets.append(dict(x=x.to(dev), ao=ao.to(dev), s_in=s_in.to(dev), wq1=wq1, sw1=sw1, wq2=wq2, sw2=sw2,
+                         y1=torch.empty((M_TOK, N_QKV), dtype=torch.bfloat16, device=dev),
+                         y2=torch.empty((M_TOK, N_O), dtype=torch.bfloat16, device=dev),
+                         ws1=B.new_workspace(B.OP_LINEAR, M_TOK, N_QKV, HID, dev),
+                         ws2=B.new_workspace(B.OP_LINEAR, M_TOK, N_O, HID, dev),
+                         hx=x.pin_memory(), hao=ao.pin_memory()))
+    qp_x, qp_o = B.QParams(4, True, 0.45, 0), B.QParams(4, True, 2.0, 0)
+    set_bytes = sum(t.numel() * t.element_size() for t in sets[0].values() if isinstance(t, torch.Tensor) and t.is_cuda)
+
+    def step(S):
+        B.fpt_w4a4_linear(S["x"], S["wq1"], S["sw1"], qp_x, B.RMSNORM, EPS, want_s_out=False, ws=S["ws1"], Y=S["y1"])
+        B.fpt_w4a4_linear(S["ao"], S["wq2"], S["sw2"], qp_o, B.SCALE_INPUT, EPS, s_in=S["s_in"], want_s_out=False,
+                          ws=S["ws2"], Y=S["y2"])
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(args.warmup, 3)):
+        step(sets[i % NSETS])
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        step(sets[i % NSETS])
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.result()
+    for S in sets:
+        assert B.fpt_check_status(S["ws1"]) == B.OK and B.fpt_check_status(S["ws2"]) == B.OK
+    if world > 1:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_per_step = ms / args.steps
+    tops = world * step_ops("attn") / (ms_per_step * 1e-3) / 1e12
+
+    # ---- end to end: host buffers in, results back, every step ------------------------------
+    h_y1 = torch.empty((M_TOK, N_QKV), dtype=torch.bfloat16).pin_memory()
+    h_y2 = torch.empty((M_TOK, N_O), dtype=torch.bfloat16).pin_memory()
+    e2e_steps = max(3, min(args.steps, 50))
+
+    def e2e_step(S):
+        S["x"].copy_(S["hx"], non_blocking=True)
+        S["ao"].copy_(S["hao"], non_blocking=True)
+        step(S)
+        h_y1.copy_(S["y1"], non_blocking=True)
+        h_y2.copy_(S["y2"], non_blocking=True)
+
+    for i in range(3):
+        e2e_step(sets[i % NSETS])
+    barrier()
+    e0.record()
+    for i in range(e2e_steps):
+        e2e_step(sets[i % NSETS])
+    e1.record()
+    barrier()
+    ms_e2e = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([ms_e2e], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item())
+    e2e_tops = world * step_ops("attn") / (ms_e2e / e2e_steps * 1e-3) / 1e12
+    h2d = 2 * M_TOK * HID * 2
+    d2h = M_TOK * (N_QKV + N_O) * 2
+
+    # ---- per-kernel pass: the same step as separate C-ABI calls with events around each -------
+    ksteps = max(8, min(args.steps, 200))
+    names = ["act_quant_x", "gemm_qkv", "act_quant_ao", "gemm_o"]
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(ksteps)]
+    xq = [torch.empty((M_TOK, HID // 2), dtype=torch.uint8, device=dev) for _ in range(2)]
+    gws = B.new_workspace(B.OP_GEMM, M_TOK, N_QKV, HID, dev)
+    for i in range(ksteps + 3):
+        S = sets[i % NSETS]
+        ev = evs[max(i - 3, 0)]
+        ev[0].record()
+        B.fpt_act_quant(S["x"], qp_x, B.RMSNORM, EPS, want_s_out=False, out=xq[0])
+        ev[1].record()
+        B.fpt_w4a4_gemm(xq[0], S["wq1"], S["sw1"], qp_x.scale, ws=gws, Y=S["y1"])
+        ev[2].record()
+        B.fpt_act_quant(S["ao"], qp_o, B.SCALE_INPUT, EPS, s_in=S["s_in"], want_s_out=False, out=xq[1])
+        ev[3].record()
+        B.fpt_w4a4_gemm(xq[1], S["wq2"], S["sw2"], qp_o.scale, ws=gws, Y=S["y2"])
+        ev[4].record()
+    torch.cuda.synchronize()
+    kern_us = {n: float(np.mean([ev[j].elapsed_time(ev[j + 1]) for ev in evs])) * 1e3 for j, n in enumerate(names)}
+    peaks = load_peaks()
+    long_run = ms > 2000.0
+    bf16_peak = peaks["bf16_sustained"] if long_run else peaks["bf16_burst"]
+    int8_peak = 2.0 * bf16_peak                       # nominal dense ratio int8 : bf16 = 4.5 : 2.25
+    gemm_ops = 2.0 * M_TOK * HID * N_QKV
+    achieved = gemm_ops / (kern_us["gemm_qkv"] * 1e-6) / 1e12
+    aq_bytes = M_TOK * HID * 2.5 + M_TOK * 4
+    roofline = {"kernel": "gemm_w4a4_kernel<256> (fused QKV, 2048x6144x4096)", "bound": "tensor",
+                "achieved": achieved, "peak": int8_peak, "unit": "TOP/s", "frac": achieved / int8_peak,
+                "traffic": None,
+                "peak_note": f"2 x {peaks['source']} bf16 {'sustained' if long_run else 'burst'} peak "
+                             f"({bf16_peak} TFLOP/s); nominal dense int8 is 4500",
+                "frac_of_nominal_4500": achieved / 4500.0,
+                "act_quant": {"bound": "hbm", "achieved": aq_bytes / (kern_us["act_quant_x"] * 1e-6) / 1e9,
+                              "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                              "frac": aq_bytes / (kern_us["act_quant_x"] * 1e-6) / 1e9 / peaks["hbm_gbs"]}}
+
+    if rank == 0:
+        rows = M_TOK
+        cpu_tops, cpu_dt = time_oracle(rows, 8)
+        line = {"metric": METRIC, "value": tops, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "int4 x int4 -> int32, scales f32, out bf16",
+                "data": "synthetic",
+                "config": {"workload": "configs[1]: Llama-3-8B-shaped attention projections, 2048 tokens, hidden "
+                                       "4096, fused QKV (6144) + O (4096), W4A4 static, per-token scale",
+                           "tokens": M_TOK, "ops_per_step": step_ops("attn"),
+                           "l2": f"rotating {NSETS} input/weight/output sets of {set_bytes / 1e6:.0f} MB each "
+                                 f"(> 126 MB L2 in total)"},
+                "e2e": {"value": e2e_tops, "unit": "TOPS", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                        "steps": e2e_steps},
+                "gpu_launches": 4 * args.steps, "clocks": clocks, "roofline": roofline,
+                "kernel_us": kern_us,
+                "cpu_baseline": {"value": cpu_tops, "unit": "TOPS", "cores": blas_threads(), "kind": "oracle",
+                                 "sample": f"{rows} of {M_TOK} token rows x all {N_QKV + N_O} output columns, "
+                                           f"8 repetitions, {cpu_dt:.2f} s each"}}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

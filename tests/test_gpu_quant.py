@@ -45,9 +45,11 @@ def test_act_quant_strided_rows_and_edge_values():
     x[4, :K] = 3.0e38                                # squares overflow float32
     qp = B.QParams(4, True, 0.41, 0)
     xq, s_out = B.fpt_act_quant(dev(x), qp, B.RMSNORM, 1e-6, K=K)
-    codes, so, _, _ = OQ.act_quant(synth.f32(x)[:, :K], oqp(qp), True, False, 1e-6)
+    with np.errstate(all="ignore"):
+        codes, so, _, _ = OQ.act_quant(synth.f32(x)[:, :K], oqp(qp), True, False, 1e-6)
     assert np.array_equal(host(xq), OQ.pack_int4(codes))
-    assert np.array_equal(host(s_out).view(np.uint32), so.view(np.uint32))
+    assert np.array_equal(host(s_out), so, equal_nan=True)           # NaN payloads may differ
+    assert np.isnan(so[2]) and so[3] == 0.0 and so[4] == 0.0
 
 
 @pytest.mark.parametrize("M,K", [(64, 1024), (7, 14336), (3, 256)])
