@@ -1,0 +1,118 @@
+"""Times one entry point of the library on one shape, with CUDA events.
+
+    python -m paper_2506_04985_b200.microbench gemm      --M 2048 --N 6144 --K 4096
+    python -m paper_2506_04985_b200.microbench act_quant --M 2048 --K 4096
+    python -m paper_2506_04985_b200.microbench silu_quant --M 4096 --K 14336
+    python -m paper_2506_04985_b200.microbench linear    --M 64 --N 14336 --K 4096
+    python -m paper_2506_04985_b200.microbench mlp       --M 4096 --K 4096 --N 14336
+
+Operands are random packed codes / random bf16 values made on the device (timing does
+not depend on the values).  `--sets S` rotates S independent operand sets so that every
+launch reads HBM rather than the L2 (pick S so that S x bytes-per-set exceeds 126 MB);
+`--reps R` launches are timed back to back between two events on the launching stream.
+Prints one JSON line: microseconds per launch, TOP/s, GB/s of algorithmic bytes.
+The same command with small `--reps` is what the profiler captures.
+"""
+import argparse
+import json
+
+import torch
+
+from . import binding as B
+
+
+def _codes(rows, kb, dev):
+    return torch.randint(0, 256, (rows, kb), dtype=torch.uint8, device=dev)
+
+
+def _bf16(rows, cols, dev):
+    return torch.randn((rows, cols), dtype=torch.float32, device=dev).to(torch.bfloat16)
+
+
+def make_case(kind, M, N, K, sets, dev, f16_scales=False):
+    """Returns (list of zero-argument launchers, algorithmic ops, algorithmic bytes)."""
+    sdt = torch.float16 if f16_scales else torch.float32
+    ssz = 2 if f16_scales else 4
+    qp = B.QParams(4, True, 0.45, 0)
+    runs = []
+    if kind == "gemm":
+        ws = B.new_workspace(B.OP_GEMM, M, N, K, dev)
+        for _ in range(sets):
+            xq, wq = _codes(M, K // 2, dev), _codes(N, K // 2, dev)
+            sw = torch.rand((N,), device=dev).to(sdt) * 0.01 + 0.001
+            y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+            runs.append(lambda xq=xq, wq=wq, sw=sw, y=y: B.fpt_w4a4_gemm(xq, wq, sw, 0.45, ws=ws, Y=y))
+        return runs, 2.0 * M * N * K, M * K / 2 + N * K / 2 + N * ssz + 2.0 * M * N
+    if kind == "act_quant":
+        for _ in range(sets):
+            x = _bf16(M, K, dev)
+            out = torch.empty((M, K // 2), dtype=torch.uint8, device=dev)
+            runs.append(lambda x=x, out=out: B.fpt_act_quant(x, qp, B.RMSNORM, 1e-5, out=out))
+        return runs, 0.0, 2.5 * M * K + 4.0 * M
+    if kind == "silu_quant":
+        for _ in range(sets):
+            gu = _bf16(M, 2 * K, dev)
+            s = torch.rand((M,), device=dev) + 0.5
+            out = torch.empty((M, K // 2), dtype=torch.uint8, device=dev)
+            runs.append(lambda gu=gu, s=s, out=out: B.fpt_act_quant(
+                gu, qp, B.SILU_MUL | B.GU_INTERLEAVED | B.SCALE_INPUT, 0.0, s_in=s, K=K, want_s_out=False, out=out))
+        return runs, 0.0, 4.5 * M * K + 4.0 * M
+    if kind == "linear":
+        for _ in range(sets):
+            x, wq = _bf16(M, K, dev), _codes(N, K // 2, dev)
+            sw = torch.rand((N,), device=dev).to(sdt) * 0.01 + 0.001
+            y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+            ws = B.new_workspace(B.OP_LINEAR, M, N, K, dev)
+            runs.append(lambda x=x, wq=wq, sw=sw, y=y, ws=ws: B.fpt_w4a4_linear(
+                x, wq, sw, qp, B.RMSNORM, 1e-5, want_s_out=False, ws=ws, Y=y))
+        return runs, 2.0 * M * N * K, 2.0 * M * K + N * K / 2 + N * ssz + 2.0 * M * N
+    if kind == "mlp":                      # K = d, N = d_ff
+        d, dff = K, N
+        for _ in range(sets):
+            x = _bf16(M, d, dev)
+            wgu, wd = _codes(2 * dff, d // 2, dev), _codes(d, dff // 2, dev)
+            sgu = torch.rand((2 * dff,), device=dev).to(sdt) * 0.01 + 0.001
+            sd = torch.rand((d,), device=dev).to(sdt) * 0.01 + 0.001
+            y = torch.empty((M, d), dtype=torch.bfloat16, device=dev)
+            ws = B.new_workspace(B.OP_MLP, M, dff, d, dev)
+            runs.append(lambda x=x, wgu=wgu, sgu=sgu, wd=wd, sd=sd, y=y, ws=ws: B.fpt_decoder_mlp(
+                x, wgu, sgu, wd, sd, qp, qp, 1e-5, want_s_out=False, ws=ws, Y=y))
+        return runs, 6.0 * M * d * dff, 4.0 * M * d + 1.5 * d * dff + 3 * dff * ssz
+    raise ValueError(kind)
+
+
+def time_case(runs, reps, warmup=3):
+    for i in range(max(warmup, 1)):
+        runs[i % len(runs)]()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(reps):
+        runs[i % len(runs)]()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) * 1e3 / reps
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("kind", choices=["gemm", "act_quant", "silu_quant", "linear", "mlp"])
+    ap.add_argument("--M", type=int, default=2048)
+    ap.add_argument("--N", type=int, default=4096)
+    ap.add_argument("--K", type=int, default=4096)
+    ap.add_argument("--sets", type=int, default=4)
+    ap.add_argument("--reps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--f16-scales", action="store_true")
+    a = ap.parse_args()
+    B.lib()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    runs, ops, nbytes = make_case(a.kind, a.M, a.N, a.K, a.sets, dev, a.f16_scales)
+    us = time_case(runs, a.reps, a.warmup)
+    print(json.dumps({"kind": a.kind, "M": a.M, "N": a.N, "K": a.K, "sets": a.sets, "reps": a.reps,
+                      "us": us, "tops": ops / us / 1e6, "gbs": nbytes / us / 1e3}))
+
+
+if __name__ == "__main__":
+    main()
