@@ -180,6 +180,35 @@ int fpt_w4a4_linear(void* stream, const void* X, int M, int K,
                     void* Y, float* s_out, void* workspace, size_t workspace_bytes);
 
 /*
+ * fpt_w4a4_linear without a caller workspace.  (The paper has no counterpart: this is a
+ * packaging variant of fpt_w4a4_linear, same arithmetic, same results.)
+ *
+ * For callers that cannot allocate device memory: a plug-in that a host runtime calls with
+ * input and output pointers only, a serving loop whose pool was frozen at start-up, code that
+ * must not trigger the device-wide synchronisation an allocation can cause.  The scratch that
+ * fpt_w4a4_linear takes from its workspace (packed activation codes, one float per token, the
+ * status block) lives in a __device__ array inside the library, FPT_STATIC_SCRATCH_BYTES long;
+ * every GPU that loads the library holds that much until the process ends.  The call itself
+ * performs no device allocation or free of any kind.
+ *
+ * Arguments as fpt_w4a4_linear, minus workspace / workspace_bytes.
+ * Limit: 256 + roundup256(M*K/2) + roundup256(4*M) <= FPT_STATIC_SCRATCH_BYTES, otherwise
+ * FPT_ERR_WORKSPACE is returned and nothing is enqueued (e.g. 4096 tokens x 8192 features fit).
+ * First call on a device: looks up the array's device address (cudaGetSymbolAddress, with that
+ * device current) and caches it; make this first call outside any stream capture.
+ * The array is shared by every call in the process and keeps the previous call's contents;
+ * the status word is cleared on `stream` at the start of each call.  Two calls that can
+ * overlap on the GPU (different streams, no dependency) race on it: serialise them.
+ * A bounded device-side wait that gave up cannot be read back through this entry point; use
+ * fpt_w4a4_linear with a workspace where that matters.
+ */
+#define FPT_STATIC_SCRATCH_BYTES (17u * 1024u * 1024u)
+int fpt_w4a4_linear_static(void* stream, const void* X, int M, int K,
+                           const uint8_t* Wq, const void* sw, int scale_dtype, const int32_t* wsum, int N,
+                           const fpt_qparams* act_qp, int flags, float eps, const float* s_in,
+                           int post_mode, const float* post, void* Y, float* s_out);
+
+/*
  * One SwiGLU MLP block in the normalised-residual form of Sec. 3.1.3:
  *   X~ = RMSNorm(X),  S_n = S_{n-1} * r                       (X is Z~_{n-1}; Eq. 7)
  *   g, u = W4A4 linears of X~ (bf16)                          grid qp_in

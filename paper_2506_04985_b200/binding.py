@@ -22,7 +22,7 @@ POST_NONE, POST_INVERSE_OF_PRE, POST_VECTOR = 0, 1, 2
 OP_LINEAR, OP_MLP, OP_GEMM = 0, 1, 2
 
 EXPORTS = ["fpt_version", "fpt_strerror", "fpt_quantize_weights", "fpt_interleave_gate_up", "fpt_act_quant",
-           "fpt_w4a4_gemm", "fpt_w4a4_linear", "fpt_decoder_mlp", "fpt_workspace_bytes", "fpt_reset_status",
+           "fpt_w4a4_gemm", "fpt_w4a4_linear", "fpt_w4a4_linear_static", "fpt_decoder_mlp", "fpt_workspace_bytes", "fpt_reset_status",
            "fpt_check_status"]
 
 
@@ -61,6 +61,7 @@ def lib():
         L.fpt_act_quant.argtypes = [vp, vp, ci, ci, ci, qp, ci, cf, vp, vp, vp, vp]
         L.fpt_w4a4_gemm.argtypes = [vp, vp, vp, ci, ci, ci, vp, ci, vp, cf, ci, ci, vp, vp, vp, vp, vp, vp, sz]
         L.fpt_w4a4_linear.argtypes = [vp, vp, ci, ci, vp, vp, ci, vp, ci, qp, ci, cf, vp, ci, vp, vp, vp, vp, sz]
+        L.fpt_w4a4_linear_static.argtypes = [vp, vp, ci, ci, vp, vp, ci, vp, ci, qp, ci, cf, vp, ci, vp, vp, vp]
         L.fpt_decoder_mlp.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp, vp, ci, qp, qp, cf, vp, vp, ci, vp, vp, sz]
         L.fpt_workspace_bytes.restype = sz
         L.fpt_workspace_bytes.argtypes = [ci, ci, ci, ci]
@@ -179,6 +180,23 @@ def fpt_w4a4_linear(X, Wq, sw, qp, flags=RMSNORM, eps=1e-5, s_in=None, post_mode
     _check(lib().fpt_w4a4_linear(_stream(), _ptr(X), M, K, _ptr(Wq), _ptr(sw), _scale_dtype(sw), _ptr(wsum), N,
                                  ctypes.byref(qp), flags, eps, _ptr(s_in), post_mode, _ptr(post), _ptr(Y),
                                  _ptr(s_out), _ptr(ws), ws.numel()), "fpt_w4a4_linear")
+    return Y, s_out
+
+
+STATIC_SCRATCH_BYTES = 17 * 1024 * 1024
+
+
+def fpt_w4a4_linear_static(X, Wq, sw, qp, flags=RMSNORM, eps=1e-5, s_in=None, post_mode=POST_NONE, post=None,
+                           wsum=None, Y=None, s_out=None):
+    """fpt_w4a4_linear on the library's built-in scratch: the call allocates nothing, so the
+    caller passes every output (Y bf16 [M, N]; s_out f32 [M] or None).  For callers that cannot
+    allocate device memory; M x K is limited by STATIC_SCRATCH_BYTES and calls must not overlap
+    on the GPU.  Returns (Y, s_out)."""
+    M, K = X.shape
+    N = Wq.shape[0]
+    _check(lib().fpt_w4a4_linear_static(_stream(), _ptr(X), M, K, _ptr(Wq), _ptr(sw), _scale_dtype(sw), _ptr(wsum),
+                                        N, ctypes.byref(qp), flags, eps, _ptr(s_in), post_mode, _ptr(post), _ptr(Y),
+                                        _ptr(s_out)), "fpt_w4a4_linear_static")
     return Y, s_out
 
 
