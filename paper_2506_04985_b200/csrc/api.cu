@@ -80,7 +80,8 @@ extern "C" int fpt_w4a4_gemm(void* stream, const uint8_t* Xq, const uint8_t* Wq,
   if (scale_dtype != FPT_DTYPE_F32 && scale_dtype != FPT_DTYPE_F16) return FPT_ERR_BAD_ARG;
   if (!(act_scale > 0.0f)) return FPT_ERR_BAD_ARG;
   if (!act_symmetric && (!wsum || act_zero_point < 0 || act_zero_point > 15)) return FPT_ERR_BAD_ARG;
-  if (((uintptr_t)Xq | (uintptr_t)Wq | (uintptr_t)Y | (uintptr_t)acc_out | (uintptr_t)residual | (uintptr_t)workspace) & 15)
+  if (((uintptr_t)Xq | (uintptr_t)Wq | (uintptr_t)Y | (uintptr_t)acc_out | (uintptr_t)residual | (uintptr_t)workspace |
+       (uintptr_t)sw | (uintptr_t)wsum) & 15)
     return FPT_ERR_ALIGNMENT;
   if (!workspace || workspace_bytes < fpt_workspace_bytes(FPT_OP_GEMM, M, N, K)) return FPT_ERR_WORKSPACE;
   GemmParams P{};

@@ -30,4 +30,7 @@ cudaError_t act_quant_launch(cudaStream_t st, const void* X, int M, int K, int l
 // gemm_w4a4.cu: validated arguments only; returns an FPT_* code.
 int gemm_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, const GemmParams& P);
 
+// gemm_w4a4_2cta.cu: the CTA-pair kernel (256 x 256 tiles) behind gemm_launch for prefill sizes.
+int gemm_pair_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, const GemmParams& P);
+
 }  // namespace fpt

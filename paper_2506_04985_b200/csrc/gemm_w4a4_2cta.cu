@@ -1,0 +1,401 @@
+// Steps (2)+(3) of the path for prefill sizes: packed-INT4 x packed-INT4 matmul with an exact
+// INT32 accumulator (App. J "Setup") and the floating-point scale factors applied after it
+// (App. B "Static quantization"), on CTA pairs.
+//
+// Why this shape: the shared-memory data pipe of an SM moves 128 bytes per cycle and is shared
+// by ld/st.shared, TMA writes and the tensor core's operand reads.  Widening nibbles to int8 in
+// shared memory for both operands of a 1-CTA tile needs 1152 of those transfers per 128-code
+// k-block against 512 cycles of MMA.  Here
+//   * two CTAs form one 256 x 256 tile (tcgen05.mma.cta_group::2): each CTA widens and feeds only
+//     its own 128 weight rows, and its tensor core reads only those;
+//   * the activation operand is widened in registers and written to TENSOR memory (tcgen05.st);
+//     the MMA takes it from there, so it is never stored to or read from shared memory as int8.
+// Per k-block and CTA: TMA in 16 KB, converter loads 16 KB, int8 weight stores 16 KB, tensor-core
+// reads 16 KB = 512 transfers for 512 MMA cycles.
+//
+// Roles per CTA (20 warps):
+//   warp 0        TMA producer: packed tiles (128 rows x 64 bytes of each operand per k-block)
+//   warp 1        tensor-memory owner; in the leader CTA (rank 0) also the MMA issuer
+//   warps 4..7    activation converters: shared -> registers -> widen -> tcgen05.st (one row per thread)
+//   warps 8..11   weight converters: shared -> widen -> 128-byte-swizzled K-major int8 tile
+//   warps 12..19  epilogue: tcgen05.ld, >> 8, scales, bf16, global stores
+// Both operands are widened as code*16 (see gemm_w4a4.cu), so the accumulator holds 256 * sum.
+#include <cuda.h>
+
+#include "fpt_internal.cuh"
+
+namespace fpt {
+namespace pair {
+
+constexpr int TM = 256, TN = 256;          // output tile of a CTA pair
+constexpr int HR = 128;                    // rows of each operand a CTA owns
+constexpr int BK = 128;                    // codes per k-block
+constexpr int PK_ROW = BK / 2;             // packed bytes per row and k-block
+constexpr int I8_ROW = BK;                 // int8 bytes per row and k-block
+constexpr int kAccCols = 256;              // tensor-memory columns of the accumulator
+constexpr int kAStageCols = BK / 4;        // 32 columns hold 128 int8 per lane
+constexpr int kTmemCols = 512;
+constexpr int kThreads = 640;
+constexpr int kConvAWarp0 = 4, kConvBWarp0 = 8, kEpiWarp0 = 12, kEpiWarps = 8;
+
+// NS: stages of widened operands (int8 weight tile in shared memory + activation columns in
+// tensor memory); NPK: stages of packed tiles in flight from TMA.
+template <int NS, int NPK>
+struct Smem {
+  static_assert(kAccCols + NS * kAStageCols <= kTmemCols, "operand stages must fit beside the accumulator");
+  static constexpr int kB8Stage = HR * I8_ROW;                      // 16 KB
+  static constexpr int kPkOp = HR * PK_ROW;                         // 8 KB
+  static constexpr int kB8Off = 0;
+  static constexpr int kPkAOff = kB8Off + NS * kB8Stage;
+  static constexpr int kPkBOff = kPkAOff + NPK * kPkOp;
+  static constexpr int kBarOff = kPkBOff + NPK * kPkOp;
+  static constexpr int kNumBars = 2 * NPK + 2 * NS + 2;
+  static constexpr int kMiscOff = kBarOff + kNumBars * 8;           // tmem base, abort flag
+  static constexpr int kBytes = kMiscOff + 16;
+  static constexpr int kAlloc = kBytes + 1024;                      // slack to align the base to 1024
+  static_assert(kAlloc <= 232448, "exceeds the shared memory of one CTA");
+};
+
+__device__ __forceinline__ void widen(const uint4& p, uint32_t* out) {      // 32 codes -> 32 int8 (x16)
+  out[0] = (p.x << 4) & 0xF0F0F0F0u;  out[4] = p.x & 0xF0F0F0F0u;
+  out[1] = (p.y << 4) & 0xF0F0F0F0u;  out[5] = p.y & 0xF0F0F0F0u;
+  out[2] = (p.z << 4) & 0xF0F0F0F0u;  out[6] = p.z & 0xF0F0F0F0u;
+  out[3] = (p.w << 4) & 0xF0F0F0F0u;  out[7] = p.w & 0xF0F0F0F0u;
+}
+
+__device__ __forceinline__ void load_scales8(const void* sw, int scale_dtype, int n, float (&o)[8]) {
+  if (scale_dtype == FPT_DTYPE_F16) {
+    const uint4 h = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const __half*>(sw) + n));
+    const __half2* h2 = reinterpret_cast<const __half2*>(&h);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { const float2 f = __half22float2(h2[j]); o[2 * j] = f.x; o[2 * j + 1] = f.y; }
+  } else {
+    const float4 a = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(sw) + n));
+    const float4 b = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(sw) + n + 4));
+    o[0] = a.x; o[1] = a.y; o[2] = a.z; o[3] = a.w; o[4] = b.x; o[5] = b.y; o[6] = b.z; o[7] = b.w;
+  }
+}
+
+template <int NS, int NPK>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                      const GemmParams P) {
+  using L = Smem<NS, NPK>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const uint32_t sbase = smem_u32(smem);
+  const uint32_t bar0 = sbase + L::kBarOff;
+  auto pk_full = [&](int s) { return bar0 + 8u * s; };
+  auto pk_empty = [&](int s) { return bar0 + 8u * (NPK + s); };
+  auto op_full = [&](int s) { return bar0 + 8u * (2 * NPK + s); };             // waited on in the leader CTA
+  auto op_empty = [&](int s) { return bar0 + 8u * (2 * NPK + NS + s); };
+  const uint32_t acc_full = bar0 + 8u * (2 * NPK + 2 * NS);
+  const uint32_t acc_empty = acc_full + 8u;                                    // waited on in the leader CTA
+  volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(smem + L::kMiscOff);
+  volatile uint32_t* abort_flag = misc + 1;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();             // 0 = leader
+  const int pair_id = blockIdx.x >> 1;
+  const int num_pairs = gridDim.x >> 1;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < NPK; ++s) { mbar_init(pk_full(s), 1); mbar_init(pk_empty(s), 8); }
+    for (int s = 0; s < NS; ++s) { mbar_init(op_full(s), 16); mbar_init(op_empty(s), 1); }
+    mbar_init(acc_full, 1);
+    mbar_init(acc_empty, 2 * kEpiWarps);
+    misc[1] = 0;
+    fence_mbar_init();
+    prefetch_tmap(&tmA);
+    prefetch_tmap(&tmB);
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(sbase + L::kMiscOff, kTmemCols);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  cluster_sync_all();                                  // barriers of both CTAs exist before any remote arrive
+  tc_fence_after();
+  const uint32_t tmem_base = misc[0];
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int s = 0; uint32_t ph = 0;
+      uint32_t armed = 0, armed_par = 0;
+      bool ok = true;
+      for (int tile = pair_id; ok && tile < P.num_tiles; tile += num_pairs) {
+        const int m0 = (tile % P.tiles_m) * TM + (int)rank * HR;
+        const int n0 = (tile / P.tiles_m) * TN + (int)rank * HR;
+        for (int kb = 0; kb < P.kblocks; ++kb) {
+          if (!mbar_wait(pk_empty(s), ph ^ 1u, abort_flag, P.status, 1)) { ok = false; break; }
+          mbar_arrive_expect_tx(pk_full(s), 2 * L::kPkOp);
+          tma_load_2d(sbase + L::kPkAOff + s * L::kPkOp, &tmA, pk_full(s), kb * PK_ROW, m0);
+          tma_load_2d(sbase + L::kPkBOff + s * L::kPkOp, &tmB, pk_full(s), kb * PK_ROW, n0);
+          armed |= 1u << s;
+          armed_par = (armed_par & ~(1u << s)) | (ph << s);
+          if (++s == NPK) { s = 0; ph ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // bounded wait for the copies still in flight before this CTA's shared memory goes away
+        const uint64_t t0 = globaltimer_ns();
+        for (int q = 0; q < NPK; ++q)
+          if (armed & (1u << q))
+            while (!mbar_try_wait(pk_full(q), (armed_par >> q) & 1u) && globaltimer_ns() - t0 < 2000000ull) {}
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (rank == 0 && lane == 0) {
+      const uint32_t idesc = umma_idesc_i8(TM, TN, !P.a_unsigned, true);
+      int s = 0; uint32_t ph = 0; int it = 0;
+      for (int tile = pair_id; tile < P.num_tiles; tile += num_pairs, ++it) {
+        if (!mbar_wait_cluster(acc_empty, (it & 1) ^ 1u, abort_flag, P.status, 2)) break;
+        tc_fence_after();
+        bool ok = true;
+        for (int kb = 0; kb < P.kblocks; ++kb) {
+          if (!mbar_wait_cluster(op_full(s), ph, abort_flag, P.status, 3)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t bdesc = umma_desc_kmajor_sw128(sbase + L::kB8Off + s * L::kB8Stage);
+          const uint32_t a_tmem = tmem_base + kAccCols + s * kAStageCols;
+#pragma unroll
+          for (int kk = 0; kk < BK / 32; ++kk)
+            umma_i8_ts_pair(tmem_base, a_tmem + 8u * kk, bdesc + 2u * kk, idesc, (kb | kk) != 0);
+          umma_commit_pair(op_empty(s), 3);
+          if (++s == NS) { s = 0; ph ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit_pair(acc_full, 3);
+      }
+    }
+  } else if (warp >= kConvAWarp0 && warp < kConvBWarp0) {
+    // ------------------------------------------------------------------ activation converters -> tensor memory
+    const int quad = warp - kConvAWarp0;                 // == warp % 4: the TMEM lanes this warp may touch
+    const int r = quad * 32 + lane;                      // row of the CTA's 128
+    const uint32_t swz = (uint32_t)((r >> 1) & 3);       // SWIZZLE_64B: 16-byte chunk index ^= (row / 2) % 4
+    const uint32_t op_full_leader = map_to_cta(op_full(0), 0);
+    int ps = 0, s = 0; uint32_t pph = 0, ph = 0;
+    bool ok = true;
+    for (int tile = pair_id; ok && tile < P.num_tiles; tile += num_pairs) {
+      for (int kb = 0; kb < P.kblocks; ++kb) {
+        if (!mbar_wait(pk_full(ps), pph, abort_flag, P.status, 5)) { ok = false; break; }
+        const uint8_t* src = smem + L::kPkAOff + ps * L::kPkOp + r * PK_ROW;
+        uint4 c[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) c[j] = *reinterpret_cast<const uint4*>(src + (((uint32_t)j ^ swz) << 4));
+        uint32_t v[32];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) widen(c[j], v + 8 * j);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(pk_empty(ps));
+        if (!mbar_wait(op_empty(s), ph ^ 1u, abort_flag, P.status, 6)) { ok = false; break; }
+        tc_fence_after();
+        tmem_st_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + kAccCols + s * kAStageCols, v);
+        tmem_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(op_full_leader + 8u * s);
+        if (++ps == NPK) { ps = 0; pph ^= 1u; }
+        if (++s == NS) { s = 0; ph ^= 1u; }
+      }
+    }
+  } else if (warp >= kConvBWarp0 && warp < kEpiWarp0) {
+    // ------------------------------------------------------------------ weight converters -> shared int8 tile
+    const int ctid = threadIdx.x - kConvBWarp0 * 32;     // 0..127
+    const uint32_t op_full_leader = map_to_cta(op_full(0), 0);
+    int ps = 0, s = 0; uint32_t pph = 0, ph = 0;
+    bool ok = true;
+    for (int tile = pair_id; ok && tile < P.num_tiles; tile += num_pairs) {
+      for (int kb = 0; kb < P.kblocks; ++kb) {
+        if (!mbar_wait(pk_full(ps), pph, abort_flag, P.status, 7)) { ok = false; break; }
+        const uint4* src = reinterpret_cast<const uint4*>(smem + L::kPkBOff + ps * L::kPkOp);
+        uint4 c[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) c[i] = src[i * 128 + ctid];
+        __syncwarp();
+        if (lane == 0) mbar_arrive(pk_empty(ps));
+        if (!mbar_wait(op_empty(s), ph ^ 1u, abort_flag, P.status, 8)) { ok = false; break; }
+        uint8_t* dst = smem + L::kB8Off + s * L::kB8Stage;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int id = i * 128 + ctid;                 // 16-byte packed chunk: row id/4, chunk id%4
+          const int r = id >> 2, ch = id & 3;
+          uint32_t w[8];
+          widen(c[i], w);
+          uint8_t* rowp = dst + r * I8_ROW;
+          *reinterpret_cast<uint4*>(rowp + (((2 * ch) ^ (r & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(rowp + (((2 * ch + 1) ^ (r & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+        }
+        fence_proxy_async_smem();       // generic-proxy writes -> visible to the tensor core's async proxy
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(op_full_leader + 8u * s);
+        if (++ps == NPK) { ps = 0; pph ^= 1u; }
+        if (++s == NS) { s = 0; ph ^= 1u; }
+      }
+    }
+  } else if (warp >= kEpiWarp0) {
+    // ------------------------------------------------------------------ epilogue
+    const int quad = warp & 3;                           // TMEM lane quadrant this warp may read
+    const int half = (warp - kEpiWarp0) >> 2;            // which 128 of the 256 columns
+    const uint32_t acc_empty_leader = map_to_cta(acc_empty, 0);
+    int it = 0;
+    for (int tile = pair_id; tile < P.num_tiles; tile += num_pairs, ++it) {
+      const int m0 = (tile % P.tiles_m) * TM + (int)rank * HR;
+      const int n0 = (tile / P.tiles_m) * TN + half * 128;
+      if (!mbar_wait(acc_full, it & 1, abort_flag, P.status, 4)) break;
+      tc_fence_after();
+      const int row = m0 + quad * 32 + lane;
+      const bool row_ok = row < P.M;
+      float c = P.act_scale, rs = 1.0f;
+      if (row_ok && P.post) c = __fmul_rn(P.act_scale, __ldg(P.post + row));
+      if (row_ok && P.res_scale) rs = __ldg(P.res_scale + row);
+      const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + half * 128;
+      const size_t rowoff = (size_t)row * (size_t)P.N;
+#pragma unroll 1
+      for (int ch = 0; ch < 4; ++ch) {
+        uint32_t v[32];
+        tmem_ld_32x32(taddr + ch * 32, v);
+        tmem_wait_ld();
+        const int col0 = n0 + ch * 32;
+        if (row_ok) {
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            const int col = col0 + g * 8;
+            if (col < P.N) {
+              int a[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j) a[j] = ((int)v[g * 8 + j]) >> 8;
+              if (P.wsum) {
+                const int4 w0 = __ldg(reinterpret_cast<const int4*>(P.wsum + col));
+                const int4 w1 = __ldg(reinterpret_cast<const int4*>(P.wsum + col + 4));
+                a[0] -= P.zero_point * w0.x; a[1] -= P.zero_point * w0.y;
+                a[2] -= P.zero_point * w0.z; a[3] -= P.zero_point * w0.w;
+                a[4] -= P.zero_point * w1.x; a[5] -= P.zero_point * w1.y;
+                a[6] -= P.zero_point * w1.z; a[7] -= P.zero_point * w1.w;
+              }
+              if (P.acc_out) {
+                int4* o = reinterpret_cast<int4*>(P.acc_out + rowoff + col);
+                o[0] = make_int4(a[0], a[1], a[2], a[3]);
+                o[1] = make_int4(a[4], a[5], a[6], a[7]);
+              }
+              if (P.Y) {
+                float sc[8], y[8];
+                load_scales8(P.sw, P.scale_dtype, col, sc);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) y[j] = __fmul_rn(__fmul_rn((float)a[j], sc[j]), c);
+                if (P.residual) {
+                  const uint4 r4 = __ldg(reinterpret_cast<const uint4*>(P.residual + rowoff + col));
+                  const uint32_t rw[4] = {r4.x, r4.y, r4.z, r4.w};
+#pragma unroll
+                  for (int j = 0; j < 4; ++j) {
+                    y[2 * j]     = __fadd_rn(y[2 * j],     __fmul_rn(bf16lo_to_f32(rw[j]), rs));
+                    y[2 * j + 1] = __fadd_rn(y[2 * j + 1], __fmul_rn(bf16hi_to_f32(rw[j]), rs));
+                  }
+                }
+                uint4 o;
+                o.x = f32_to_bf16_bits(y[0]) | (f32_to_bf16_bits(y[1]) << 16);
+                o.y = f32_to_bf16_bits(y[2]) | (f32_to_bf16_bits(y[3]) << 16);
+                o.z = f32_to_bf16_bits(y[4]) | (f32_to_bf16_bits(y[5]) << 16);
+                o.w = f32_to_bf16_bits(y[6]) | (f32_to_bf16_bits(y[7]) << 16);
+                *reinterpret_cast<uint4*>(P.Y + rowoff + col) = o;
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  // Neither CTA may leave (or free tensor memory) while its peer can still arrive on its
+  // barriers or the pair's MMAs can still read its shared / tensor memory.
+  __syncwarp();
+  tc_fence_before();
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, kTmemCols);
+  }
+}
+
+// ------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// Tensor map over a packed [rows, K/2]-byte matrix; one box = 128 rows of one k-block (64 bytes each).
+static bool make_map(CUtensorMap* m, const void* base, int rows, int K, CUtensorMapSwizzle swz) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)(K / 2), (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)(K / 2)};
+  const cuuint32_t box[2] = {(cuuint32_t)PK_ROW, (cuuint32_t)HR};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int NS, int NPK>
+static int launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, GemmParams P) {
+  using L = Smem<NS, NPK>;
+  auto kern = gemm_w4a4_pair_kernel<NS, NPK>;
+  static int max_pairs = 0;                 // co-resident CTA pairs on this device
+  if (!max_pairs) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kAlloc) != cudaSuccess)
+      return FPT_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2, 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = L::kAlloc;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) {
+      cudaGetLastError();
+      int dev = 0, sms = 0;
+      cudaGetDevice(&dev);
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+      n = sms / 2;
+    }
+    max_pairs = n > 0 ? n : 1;
+  }
+  CUtensorMap tmA, tmB;
+  if (!make_map(&tmA, Xq, P.M, P.K, CU_TENSOR_MAP_SWIZZLE_64B) || !make_map(&tmB, Wq, P.N, P.K, CU_TENSOR_MAP_SWIZZLE_NONE))
+    return FPT_ERR_CUDA;
+  P.tiles_m = (P.M + TM - 1) / TM;
+  P.num_tiles = P.tiles_m * ((P.N + TN - 1) / TN);
+  P.kblocks = P.K / BK;
+  const int pairs = P.num_tiles < max_pairs ? P.num_tiles : max_pairs;
+  kern<<<2 * pairs, kThreads, L::kAlloc, st>>>(tmA, tmB, P);
+  return cudaGetLastError() == cudaSuccess ? FPT_OK : FPT_ERR_CUDA;
+}
+
+}  // namespace pair
+
+int gemm_pair_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, const GemmParams& P) {
+  return pair::launch<4, 9>(st, Xq, Wq, P);
+}
+
+}  // namespace fpt
