@@ -189,20 +189,23 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank
 }
 // Arrive on an mbarrier that may live in another CTA of the cluster (address from map_to_cta).
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+  // Default semantics (release at CTA scope): what the arriving thread publishes is already
+  // complete where it will be read (its own shared / tensor memory, fenced for the async proxy);
+  // the arrival only signals.  A cluster-scope release here costs several hundred cycles per call.
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
   uint32_t done;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(done)
       : "r"(bar), "r"(parity)
       : "memory");
   return done;
 }
-// mbar_wait for a barrier on which threads of the peer CTA arrive (acquire at cluster scope).
+// mbar_wait for a barrier on which threads of the peer CTA arrive too.
 __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
                                                   uint32_t* status, uint32_t role) {
   if (mbar_try_wait_cluster(bar, parity)) return true;
