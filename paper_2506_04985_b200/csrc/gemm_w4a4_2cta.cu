@@ -18,7 +18,8 @@
 //   warp 1        tensor-memory owner; in the leader CTA (rank 0) also the MMA issuer
 //   warps 4..7    activation converters: shared -> registers -> widen -> tcgen05.st (one row per thread)
 //   warps 8..11   weight converters: shared -> widen -> 128-byte-swizzled K-major int8 tile
-//   warps 12..19  epilogue: tcgen05.ld, >> 8, scales, bf16, global stores
+//   warps 12..19  epilogue: tcgen05.ld, >> 8, scales, bf16 into a swizzled shared-memory tile; the
+//                 accumulator is released as soon as it has been read, the tile leaves by TMA store
 // Both operands are widened as code*16 (see gemm_w4a4.cu), so the accumulator holds 256 * sum.
 #include <cuda.h>
 
@@ -48,8 +49,11 @@ struct Smem {
   static constexpr int kB8Off = 0;
   static constexpr int kPkAOff = kB8Off + NS * kB8Stage;
   static constexpr int kPkBOff = kPkAOff + NPK * kPkOp;
-  static constexpr int kBarOff = kPkBOff + NPK * kPkOp;
-  static constexpr int kNumBars = 2 * NPK + 2 * NS + 2;
+  static constexpr int kStgOff = kPkBOff + NPK * kPkOp;             // bf16 output tile: 4 slabs of 128 rows x 64 columns
+  static constexpr int kStgSlab = HR * 128;                         // 16 KB, 128-byte rows, 128-byte swizzle
+  static constexpr int kScaleOff = kStgOff + 4 * kStgSlab;          // 2 x 256 floats (sw) + 2 x 256 ints (z * wsum)
+  static constexpr int kBarOff = kScaleOff + 2 * TN * 4 * 2;
+  static constexpr int kNumBars = 2 * NPK + 2 * NS + 2 + 2 + 2 + 2;
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;           // tmem base, abort flag
   static constexpr int kBytes = kMiscOff + 16;
   static constexpr int kAlloc = kBytes + 1024;                      // slack to align the base to 1024
@@ -79,7 +83,7 @@ __device__ __forceinline__ void load_scales8(const void* sw, int scale_dtype, in
 template <int NS, int NPK>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                      const GemmParams P) {
+                      const __grid_constant__ CUtensorMap tmY, const GemmParams P) {
   using L = Smem<NS, NPK>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -91,6 +95,9 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
   auto op_empty = [&](int s) { return bar0 + 8u * (2 * NPK + NS + s); };
   const uint32_t acc_full = bar0 + 8u * (2 * NPK + 2 * NS);
   const uint32_t acc_empty = acc_full + 8u;                                    // waited on in the leader CTA
+  auto sc_full = [&](int b) { return acc_full + 16u + 8u * b; };               // scales of a tile are in shared memory
+  auto stg_full = [&](int h) { return acc_full + 32u + 8u * h; };              // a 128-column half of the tile is staged
+  auto stg_empty = [&](int h) { return acc_full + 48u + 8u * h; };             // ... and has been read by its TMA store
   volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(smem + L::kMiscOff);
   volatile uint32_t* abort_flag = misc + 1;
 
@@ -105,10 +112,12 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     for (int s = 0; s < NS; ++s) { mbar_init(op_full(s), 16); mbar_init(op_empty(s), 1); }
     mbar_init(acc_full, 1);
     mbar_init(acc_empty, 2 * kEpiWarps);
+    for (int b = 0; b < 2; ++b) { mbar_init(sc_full(b), kEpiWarps); mbar_init(stg_full(b), 4); mbar_init(stg_empty(b), 1); }
     misc[1] = 0;
     fence_mbar_init();
     prefetch_tmap(&tmA);
     prefetch_tmap(&tmB);
+    if (P.Y) prefetch_tmap(&tmY);
   }
   if (warp == 1) {
     tmem_alloc_pair(sbase + L::kMiscOff, kTmemCols);
@@ -239,76 +248,105 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     // ------------------------------------------------------------------ epilogue
     const int quad = warp & 3;                           // TMEM lane quadrant this warp may read
     const int half = (warp - kEpiWarp0) >> 2;            // which 128 of the 256 columns
+    const int etid = (warp - kEpiWarp0) * 32 + lane;     // 0..255: the tile column whose scale this thread fetches
     const uint32_t acc_empty_leader = map_to_cta(acc_empty, 0);
+    float* sw_s = reinterpret_cast<float*>(smem + L::kScaleOff);
+    int* zw_s = reinterpret_cast<int*>(smem + L::kScaleOff + 2 * TN * 4);
+    const int r = quad * 32 + lane;                      // row of the CTA's 128
+    const bool magic_ok = P.K <= 32768;                  // |acc| < 2^22: int -> float by exponent trick
+    const bool issuer = quad == 0 && lane == 0;          // issues the TMA stores of its half
     int it = 0;
     for (int tile = pair_id; tile < P.num_tiles; tile += num_pairs, ++it) {
+      const int b = it & 1; const uint32_t bph = (it >> 1) & 1;
       const int m0 = (tile % P.tiles_m) * TM + (int)rank * HR;
-      const int n0 = (tile / P.tiles_m) * TN + half * 128;
-      if (!mbar_wait(acc_full, it & 1, abort_flag, P.status, 4)) break;
-      tc_fence_after();
-      const int row = m0 + quad * 32 + lane;
+      const int nt = (tile / P.tiles_m) * TN;            // first column of the tile
+      // scale factors of the tile's columns -> shared memory, while the matmul of the tile runs
+      {
+        const int n = nt + etid;
+        sw_s[b * TN + etid] = n < P.N ? load_scale(P.sw, P.scale_dtype, n) : 0.0f;
+        zw_s[b * TN + etid] = (P.wsum && n < P.N) ? P.zero_point * __ldg(P.wsum + n) : 0;
+      }
+      const int row = m0 + r;
       const bool row_ok = row < P.M;
       float c = P.act_scale, rs = 1.0f;
       if (row_ok && P.post) c = __fmul_rn(P.act_scale, __ldg(P.post + row));
       if (row_ok && P.res_scale) rs = __ldg(P.res_scale + row);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(sc_full(b));
+      if (!mbar_wait(sc_full(b), bph, abort_flag, P.status, 9)) break;
+      // the staging half must have been read by the TMA store of the previous tile
+      if (P.Y && !mbar_wait(stg_empty(half), (it & 1) ^ 1u, abort_flag, P.status, 10)) break;
+      if (!mbar_wait(acc_full, it & 1, abort_flag, P.status, 4)) break;
+      tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + half * 128;
       const size_t rowoff = (size_t)row * (size_t)P.N;
+      const float* sws = sw_s + b * TN + half * 128;
+      const int* zws = zw_s + b * TN + half * 128;
 #pragma unroll 1
       for (int ch = 0; ch < 4; ++ch) {
         uint32_t v[32];
         tmem_ld_32x32(taddr + ch * 32, v);
         tmem_wait_ld();
-        const int col0 = n0 + ch * 32;
-        if (row_ok) {
+        uint8_t* slab = smem + L::kStgOff + (half * 2 + (ch >> 1)) * L::kStgSlab + r * 128;
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            const int col = col0 + g * 8;
-            if (col < P.N) {
-              int a[8];
+        for (int g = 0; g < 4; ++g) {
+          const int col = nt + half * 128 + ch * 32 + g * 8;
+          int a[8];
 #pragma unroll
-              for (int j = 0; j < 8; ++j) a[j] = ((int)v[g * 8 + j]) >> 8;
-              if (P.wsum) {
-                const int4 w0 = __ldg(reinterpret_cast<const int4*>(P.wsum + col));
-                const int4 w1 = __ldg(reinterpret_cast<const int4*>(P.wsum + col + 4));
-                a[0] -= P.zero_point * w0.x; a[1] -= P.zero_point * w0.y;
-                a[2] -= P.zero_point * w0.z; a[3] -= P.zero_point * w0.w;
-                a[4] -= P.zero_point * w1.x; a[5] -= P.zero_point * w1.y;
-                a[6] -= P.zero_point * w1.z; a[7] -= P.zero_point * w1.w;
-              }
-              if (P.acc_out) {
-                int4* o = reinterpret_cast<int4*>(P.acc_out + rowoff + col);
-                o[0] = make_int4(a[0], a[1], a[2], a[3]);
-                o[1] = make_int4(a[4], a[5], a[6], a[7]);
-              }
-              if (P.Y) {
-                float sc[8], y[8];
-                load_scales8(P.sw, P.scale_dtype, col, sc);
+          for (int j = 0; j < 8; ++j) a[j] = (((int)v[g * 8 + j]) >> 8) - zws[ch * 32 + g * 8 + j];
+          if (P.acc_out && row_ok && col < P.N) {
+            int4* o = reinterpret_cast<int4*>(P.acc_out + rowoff + col);
+            o[0] = make_int4(a[0], a[1], a[2], a[3]);
+            o[1] = make_int4(a[4], a[5], a[6], a[7]);
+          }
+          if (P.Y) {
+            float y[8];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) y[j] = __fmul_rn(__fmul_rn((float)a[j], sc[j]), c);
-                if (P.residual) {
-                  const uint4 r4 = __ldg(reinterpret_cast<const uint4*>(P.residual + rowoff + col));
-                  const uint32_t rw[4] = {r4.x, r4.y, r4.z, r4.w};
+            for (int j = 0; j < 8; ++j) {
+              // exact int -> float: 1.5 * 2^23 + a has a in its low mantissa bits
+              const float af = magic_ok ? __fsub_rn(__int_as_float(0x4B400000 + a[j]), 12582912.0f) : (float)a[j];
+              y[j] = __fmul_rn(__fmul_rn(af, sws[ch * 32 + g * 8 + j]), c);
+            }
+            if (P.residual && row_ok && col < P.N) {
+              const uint4 r4 = __ldg(reinterpret_cast<const uint4*>(P.residual + rowoff + col));
+              const uint32_t rw[4] = {r4.x, r4.y, r4.z, r4.w};
 #pragma unroll
-                  for (int j = 0; j < 4; ++j) {
-                    y[2 * j]     = __fadd_rn(y[2 * j],     __fmul_rn(bf16lo_to_f32(rw[j]), rs));
-                    y[2 * j + 1] = __fadd_rn(y[2 * j + 1], __fmul_rn(bf16hi_to_f32(rw[j]), rs));
-                  }
-                }
-                uint4 o;
-                o.x = f32_to_bf16_bits(y[0]) | (f32_to_bf16_bits(y[1]) << 16);
-                o.y = f32_to_bf16_bits(y[2]) | (f32_to_bf16_bits(y[3]) << 16);
-                o.z = f32_to_bf16_bits(y[4]) | (f32_to_bf16_bits(y[5]) << 16);
-                o.w = f32_to_bf16_bits(y[6]) | (f32_to_bf16_bits(y[7]) << 16);
-                *reinterpret_cast<uint4*>(P.Y + rowoff + col) = o;
+              for (int j = 0; j < 4; ++j) {
+                y[2 * j]     = __fadd_rn(y[2 * j],     __fmul_rn(bf16lo_to_f32(rw[j]), rs));
+                y[2 * j + 1] = __fadd_rn(y[2 * j + 1], __fmul_rn(bf16hi_to_f32(rw[j]), rs));
               }
             }
+            uint4 o;
+            o.x = f32_to_bf16_bits(y[0]) | (f32_to_bf16_bits(y[1]) << 16);
+            o.y = f32_to_bf16_bits(y[2]) | (f32_to_bf16_bits(y[3]) << 16);
+            o.z = f32_to_bf16_bits(y[4]) | (f32_to_bf16_bits(y[5]) << 16);
+            o.w = f32_to_bf16_bits(y[6]) | (f32_to_bf16_bits(y[7]) << 16);
+            const int chunk = (ch & 1) * 4 + g;          // 16-byte chunk of the slab row; 128-byte swizzle
+            *reinterpret_cast<uint4*>(slab + ((chunk ^ (r & 7)) << 4)) = o;
           }
         }
       }
+      // the accumulator has been read: the next tile's matmul may overwrite it
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
+      if (P.Y) {
+        fence_proxy_async_smem();                        // staged tile -> visible to the TMA engine
+        __syncwarp();
+        if (lane == 0) mbar_arrive(stg_full(half));
+        if (issuer) {
+          if (!mbar_wait(stg_full(half), it & 1, abort_flag, P.status, 11)) break;
+          const uint32_t s0 = sbase + L::kStgOff + (half * 2) * L::kStgSlab;
+          tma_store_2d(&tmY, s0, nt + half * 128, m0);
+          tma_store_2d(&tmY, s0 + L::kStgSlab, nt + half * 128 + 64, m0);
+          tma_store_commit();
+          tma_store_wait_read();
+          mbar_arrive(stg_empty(half));
+        }
+        __syncwarp();
+      }
     }
+    if (issuer) tma_store_wait_read();
   }
 
   // ------------------------------------------------------------------ teardown
@@ -355,6 +393,19 @@ static bool make_map(CUtensorMap* m, const void* base, int rows, int K, CUtensor
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tensor map over the bf16 output [M, N]; one box = 128 rows x 64 columns, 128-byte swizzle in shared memory.
+static bool make_out_map(CUtensorMap* m, const void* base, int M, int N) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
+  const cuuint64_t strides[1] = {(cuuint64_t)N * 2};
+  const cuuint32_t box[2] = {64, (cuuint32_t)HR};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int NS, int NPK>
 static int launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, GemmParams P) {
   using L = Smem<NS, NPK>;
@@ -381,21 +432,22 @@ static int launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, GemmPar
     }
     max_pairs = n > 0 ? n : 1;
   }
-  CUtensorMap tmA, tmB;
+  CUtensorMap tmA, tmB, tmY;
   if (!make_map(&tmA, Xq, P.M, P.K, CU_TENSOR_MAP_SWIZZLE_64B) || !make_map(&tmB, Wq, P.N, P.K, CU_TENSOR_MAP_SWIZZLE_NONE))
     return FPT_ERR_CUDA;
+  if (P.Y) { if (!make_out_map(&tmY, P.Y, P.M, P.N)) return FPT_ERR_CUDA; } else tmY = tmA;   // unused without Y
   P.tiles_m = (P.M + TM - 1) / TM;
   P.num_tiles = P.tiles_m * ((P.N + TN - 1) / TN);
   P.kblocks = P.K / BK;
   const int pairs = P.num_tiles < max_pairs ? P.num_tiles : max_pairs;
-  kern<<<2 * pairs, kThreads, L::kAlloc, st>>>(tmA, tmB, P);
+  kern<<<2 * pairs, kThreads, L::kAlloc, st>>>(tmA, tmB, tmY, P);
   return cudaGetLastError() == cudaSuccess ? FPT_OK : FPT_ERR_CUDA;
 }
 
 }  // namespace pair
 
 int gemm_pair_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, const GemmParams& P) {
-  return pair::launch<4, 9>(st, Xq, Wq, P);
+  return pair::launch<4, 5>(st, Xq, Wq, P);
 }
 
 }  // namespace fpt
