@@ -156,9 +156,10 @@ int fpt_act_quant(void* stream, const void* X, int M, int K, int ldx,
  *   res_scale [M] f32 or NULL (1).
  *   Y [M, N] bf16 out (may be NULL when acc_out is given)
  *   acc_out [M, N] int32 or NULL: debugging aid, the raw accumulators.
- *   workspace: fpt_workspace_bytes(FPT_OP_GEMM, M, N, K) bytes; its first word is the
- *   status word read by fpt_check_status.
- * M >= 1; K % 128 == 0; N % 8 == 0.  For M <= 64 a weight-streaming kernel is used.
+ *   workspace: fpt_workspace_bytes(FPT_OP_GEMM, M, N, K) bytes; it starts with an 8 KiB control
+ *   block (status word read by fpt_check_status, tile counters) that fpt_reset_status zeroes.
+ * M >= 1; K % 128 == 0; N % 8 == 0.  For M <= 64 a weight-streaming kernel is used: it splits
+ * the weight stream evenly over the SMs and adds the partial sums up as exact integers.
  */
 int fpt_w4a4_gemm(void* stream, const uint8_t* Xq, const uint8_t* Wq, int M, int N, int K,
                   const void* sw, int scale_dtype, const int32_t* wsum,
@@ -192,7 +193,8 @@ int fpt_w4a4_linear(void* stream, const void* X, int M, int K,
  * performs no device allocation or free of any kind.
  *
  * Arguments as fpt_w4a4_linear, minus workspace / workspace_bytes.
- * Limit: 256 + roundup256(M*K/2) + roundup256(4*M) <= FPT_STATIC_SCRATCH_BYTES, otherwise
+ * Limit: fpt_workspace_bytes(FPT_OP_LINEAR, M, N, K) <= FPT_STATIC_SCRATCH_BYTES (about
+ * M*K/2 + 4*M + 8 KiB, plus up to 10 MiB of matmul scratch when M <= 64), otherwise
  * FPT_ERR_WORKSPACE is returned and nothing is enqueued (e.g. 4096 tokens x 8192 features fit).
  * First call on a device: looks up the array's device address (cudaGetSymbolAddress, with that
  * device current) and caches it; make this first call outside any stream capture.
@@ -231,7 +233,8 @@ int fpt_decoder_mlp(void* stream, const void* X, int M, int d, int d_ff,
  * FPT_OP_LINEAR / FPT_OP_GEMM: (M, N, K); FPT_OP_MLP: (M, d_ff, d). */
 size_t fpt_workspace_bytes(int op, int M, int N, int K);
 
-/* Zeroes the status word of a workspace (call once after allocating it). */
+/* Zeroes the control block (first 8 KiB: status word, tile counters) of a workspace.  Call once
+ * after allocating it, and again after a call that ended in FPT_ERR_TIMEOUT. */
 int fpt_reset_status(void* stream, void* workspace);
 
 /* Synchronises `stream`, reads the status word at the start of `workspace` and returns

@@ -44,12 +44,13 @@ extern "C" size_t fpt_workspace_bytes(int op, int M, int N, int K) {
   const size_t m = (size_t)M;
   switch (op) {
     case FPT_OP_GEMM:
-      return kStatusBytes;
+      return kStatusBytes + gemm_scratch_bytes(M);
     case FPT_OP_LINEAR:
-      return kStatusBytes + up256(m * (size_t)K / 2) + up256(m * 4);
+      return kStatusBytes + gemm_scratch_bytes(M) + up256(m * (size_t)K / 2) + up256(m * 4);
     case FPT_OP_MLP: {   // N = d_ff, K = d
       const size_t dff = (size_t)N, d = (size_t)K;
-      return kStatusBytes + up256(m * d / 2) + 2 * up256(m * 4) + up256(m * 2 * dff * 2) + up256(m * dff / 2);
+      return kStatusBytes + gemm_scratch_bytes(M) + up256(m * d / 2) + 2 * up256(m * 4) + up256(m * 2 * dff * 2) +
+             up256(m * dff / 2);
     }
     default:
       return 0;
@@ -97,6 +98,7 @@ extern "C" int fpt_w4a4_gemm(void* stream, const uint8_t* Xq, const uint8_t* Wq,
   P.Y = reinterpret_cast<__nv_bfloat16*>(Y);
   P.acc_out = acc_out;
   P.status = reinterpret_cast<uint32_t*>(workspace);
+  P.scratch = reinterpret_cast<uint8_t*>(workspace) + kStatusBytes;
   return gemm_launch((cudaStream_t)stream, Xq, Wq, P);
 }
 
@@ -117,7 +119,8 @@ extern "C" int fpt_w4a4_linear(void* stream, const void* X, int M, int K, const 
   if (((uintptr_t)X | (uintptr_t)Wq | (uintptr_t)Y | (uintptr_t)workspace) & 15) return FPT_ERR_ALIGNMENT;
   if (!workspace || workspace_bytes < fpt_workspace_bytes(FPT_OP_LINEAR, M, N, K)) return FPT_ERR_WORKSPACE;
   uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
-  uint8_t* Xq = ws + kStatusBytes;
+  const size_t gemm_ws = kStatusBytes + gemm_scratch_bytes(M);      // control block + matmul scratch
+  uint8_t* Xq = ws + gemm_ws;
   float* post_inv = reinterpret_cast<float*>(Xq + up256((size_t)M * K / 2));
   cudaStream_t st = (cudaStream_t)stream;
   if (act_quant_launch(st, X, M, K, K, act_qp, flags, eps, nullptr, s_in, Xq, s_out,
@@ -125,7 +128,7 @@ extern "C" int fpt_w4a4_linear(void* stream, const void* X, int M, int K, const 
     return FPT_ERR_CUDA;
   const float* pv = post_mode == FPT_POST_NONE ? nullptr : post_mode == FPT_POST_VECTOR ? post : post_inv;
   return fpt_w4a4_gemm(stream, Xq, Wq, M, N, K, sw, scale_dtype, wsum, act_qp->scale, act_qp->symmetric,
-                       act_qp->zero_point, pv, nullptr, nullptr, Y, nullptr, workspace, kStatusBytes);
+                       act_qp->zero_point, pv, nullptr, nullptr, Y, nullptr, workspace, gemm_ws);
 }
 
 extern "C" int fpt_decoder_mlp(void* stream, const void* X, int M, int d, int d_ff, const uint8_t* Wgu_q,
@@ -146,7 +149,8 @@ extern "C" int fpt_decoder_mlp(void* stream, const void* X, int M, int d, int d_
   if (!workspace || workspace_bytes < fpt_workspace_bytes(FPT_OP_MLP, M, d_ff, d)) return FPT_ERR_WORKSPACE;
   const size_t m = (size_t)M;
   uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
-  uint8_t* Xq = ws + kStatusBytes;
+  const size_t gemm_ws = kStatusBytes + gemm_scratch_bytes(M);      // control block + matmul scratch
+  uint8_t* Xq = ws + gemm_ws;
   float* sn_ws = reinterpret_cast<float*>(Xq + up256(m * d / 2));
   float* r_ws = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(sn_ws) + up256(m * 4));
   uint8_t* GU = reinterpret_cast<uint8_t*>(r_ws) + up256(m * 4);
@@ -159,7 +163,7 @@ extern "C" int fpt_decoder_mlp(void* stream, const void* X, int M, int d, int d_
     return FPT_ERR_CUDA;
   // gate || up in one matmul over the interleaved weight
   rc = fpt_w4a4_gemm(stream, Xq, Wgu_q, M, 2 * d_ff, d, sw_gu, scale_dtype, nullptr, qp_in->scale, 1, 0, nullptr,
-                     nullptr, nullptr, GU, nullptr, workspace, kStatusBytes);
+                     nullptr, nullptr, GU, nullptr, workspace, gemm_ws);
   if (rc) return rc;
   // m = bf16(silu(g) * u), quantised after the multiply by S_n
   if (act_quant_launch(st, GU, M, d_ff, 2 * d_ff, qp_mid, FPT_SILU_MUL | FPT_GU_INTERLEAVED | FPT_SCALE_INPUT, 0.0f,
@@ -167,5 +171,5 @@ extern "C" int fpt_decoder_mlp(void* stream, const void* X, int M, int d, int d_
     return FPT_ERR_CUDA;
   // down projection; the normalised residual X * r joins before the final rounding
   return fpt_w4a4_gemm(stream, Mq, Wd_q, M, d, d_ff, sw_d, scale_dtype, nullptr, qp_mid->scale, 1, 0, nullptr,
-                       add_residual ? X : nullptr, add_residual ? r_ws : nullptr, Y, nullptr, workspace, kStatusBytes);
+                       add_residual ? X : nullptr, add_residual ? r_ws : nullptr, Y, nullptr, workspace, gemm_ws);
 }

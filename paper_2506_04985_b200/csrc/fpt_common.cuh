@@ -15,7 +15,11 @@ namespace fpt {
 // status word (first 4 bytes of a workspace): 0 = fine, otherwise where a wait gave up
 // ----------------------------------------------------------------------------------
 constexpr uint32_t kStatusTimeoutBase = 0x7100u;     // | role id
-constexpr size_t   kStatusBytes       = 256;         // status block at the head of a workspace
+constexpr size_t   kStatusBytes       = 8192;        // control block at the head of a workspace: status word,
+                                                      // then (from byte 256) the tile counters of the decode matmul
+constexpr int      kCounterWord0      = 64;          // first counter, in 32-bit words from the workspace start
+constexpr int      kDecodeMaxCounters = (int)(kStatusBytes / 4) - kCounterWord0;
+constexpr int      kDecodeMaxCtas     = 160;         // the decode matmul never launches more CTAs than this
 
 // ----------------------------------------------------------------------------------
 // float helpers: one rounding per operation, never contracted into an FMA

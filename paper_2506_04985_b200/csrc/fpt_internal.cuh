@@ -19,7 +19,8 @@ struct GemmParams {
   const float* res_scale;
   __nv_bfloat16* Y;
   int32_t* acc_out;
-  uint32_t* status;
+  uint32_t* status;            // control block of the workspace (status word, decode counters)
+  void* scratch;               // gemm_scratch_bytes(M) bytes behind the control block (decode partial sums)
 };
 
 // act_quant.cu: validated arguments only; also fills 1/p_t and r_t for the composed calls.
@@ -29,6 +30,11 @@ cudaError_t act_quant_launch(cudaStream_t st, const void* X, int M, int K, int l
 
 // gemm_w4a4.cu: validated arguments only; returns an FPT_* code.
 int gemm_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, const GemmParams& P);
+
+// gemm_decode.cu: the weight-streaming kernel for M <= 64 and the scratch it needs.
+size_t gemm_decode_scratch_bytes(int M);
+int gemm_decode_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, const GemmParams& P, void* scratch);
+inline size_t gemm_scratch_bytes(int M) { return M <= 64 ? gemm_decode_scratch_bytes(M) : 0; }
 
 // gemm_w4a4_2cta.cu: the CTA-pair kernel (256 x 256 tiles) behind gemm_launch for prefill sizes.
 int gemm_pair_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, const GemmParams& P);

@@ -1,0 +1,427 @@
+// Steps (2)+(3) of the path at decode sizes (at most 64 tokens): the packed INT4 weights are
+// streamed once from HBM, which is the whole cost; the arithmetic is the same exact INT32
+// matmul (App. J "Setup") and scale-factor epilogue (App. B "Static quantization").
+//
+// The operands swap sides: 128 WEIGHT rows are the M side of the MMA and the (padded) tokens
+// are its N side, so one tcgen05.mma of shape 128 x {16,32,64} x 32 consumes 128 x 32 weight
+// codes.  Weights are widened nibble -> int8 in registers and written to tensor memory
+// (tcgen05.st), the MMA reads them from there; only the few token rows are widened into a
+// shared-memory tile.  Nothing of the weight stream is ever stored to shared memory twice.
+//
+// Work is split stream-K style: the T = (N/128) * (K/128) weight k-blocks are cut into equal
+// contiguous ranges, one per CTA (one CTA per SM), so every SM streams the same number of bytes
+// whatever the shape.  A range that covers part of a tile leaves its raw int32 partial sums in
+// a scratch slot; the last CTA to arrive at a tile (an atomic counter per tile and lane
+// quadrant) adds the slots up -- integer addition, so the result does not depend on the order
+// -- and runs the epilogue.  No CTA ever waits for another.
+//
+// Roles (16 warps): warp 0 TMA producer, warp 1 MMA issuer and tensor-memory owner, warps 2-3
+// token converters, warps 4-11 weight converters (two groups taking alternate k-blocks),
+// warps 12-15 epilogue.
+#include <cuda.h>
+
+#include "fpt_internal.cuh"
+
+namespace fpt {
+namespace decode {
+
+constexpr int HR = 128;                    // weight rows per tile
+constexpr int BK = 128;                    // codes per k-block
+constexpr int PK_ROW = BK / 2;
+constexpr int I8_ROW = BK;
+constexpr int NS = 8;                      // widened stages: 8 x 32 tensor-memory columns + 8 token tiles
+constexpr int NPK = 12;                    // packed stages in flight from TMA
+constexpr int kMaxTok = 64;
+constexpr int kAccCols = 64;               // per accumulator buffer (two of them)
+constexpr int kAStage0 = 2 * kAccCols;
+constexpr int kTmemCols = 512;
+constexpr int kThreads = 512;
+constexpr int kConvBWarp0 = 2, kConvAWarp0 = 4, kEpiWarp0 = 12;
+
+struct Smem {
+  static constexpr int kB8Stage = kMaxTok * I8_ROW;                 // 8 KB: widened token tile
+  static constexpr int kPkW = HR * PK_ROW;                          // 8 KB: packed weights of one k-block
+  static constexpr int kPkX = kMaxTok * PK_ROW;                     // 4 KB: packed tokens of one k-block
+  static constexpr int kB8Off = 0;
+  static constexpr int kPkWOff = kB8Off + NS * kB8Stage;
+  static constexpr int kPkXOff = kPkWOff + NPK * kPkW;
+  static constexpr int kVecOff = kPkXOff + NPK * kPkX;              // c_t and residual scale per token: 2 x 64 floats
+  static constexpr int kBarOff = kVecOff + 2 * kMaxTok * 4;
+  static constexpr int kNumBars = 2 * NPK + 2 * NS + 4;
+  static constexpr int kMiscOff = kBarOff + kNumBars * 8;
+  static constexpr int kBytes = kMiscOff + 16;
+  static constexpr int kAlloc = kBytes + 1024;
+  static_assert(kAlloc <= 232448, "exceeds the shared memory of one CTA");
+};
+
+struct DecodeParams {
+  GemmParams g;            // M = tokens, N = weight rows, K
+  int npad;                // tokens padded to the MMA N: 16, 32 or 64
+  int tiles;               // N / 128 rounded up
+  int kblocks;             // K / 128
+  long long total;         // tiles * kblocks
+  int whole_tiles;         // 1: ranges end on tile boundaries (no partial sums, no counters)
+  int32_t* slots;          // [gridDim.x][2][npad][128] raw int32 partial sums
+  uint32_t* counters;      // [tiles][4], zero between launches
+};
+
+// First weight k-block (global index) of CTA c's range.
+__device__ __forceinline__ long long range_start(const DecodeParams& D, int c, int nctas) {
+  if (D.whole_tiles) return (long long)D.kblocks * (((long long)D.tiles * c) / nctas);
+  return (D.total * c) / nctas;
+}
+
+__device__ __forceinline__ void widen(const uint4& p, uint32_t* out) {      // 32 codes -> 32 int8 (x16)
+  out[0] = (p.x << 4) & 0xF0F0F0F0u;  out[4] = p.x & 0xF0F0F0F0u;
+  out[1] = (p.y << 4) & 0xF0F0F0F0u;  out[5] = p.y & 0xF0F0F0F0u;
+  out[2] = (p.z << 4) & 0xF0F0F0F0u;  out[6] = p.z & 0xF0F0F0F0u;
+  out[3] = (p.w << 4) & 0xF0F0F0F0u;  out[7] = p.w & 0xF0F0F0F0u;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_w4a4_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
+                        const DecodeParams D) {
+  using L = Smem;
+  const GemmParams& P = D.g;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const uint32_t sbase = smem_u32(smem);
+  const uint32_t bar0 = sbase + L::kBarOff;
+  auto pk_full = [&](int s) { return bar0 + 8u * s; };
+  auto pk_empty = [&](int s) { return bar0 + 8u * (NPK + s); };
+  auto op_full = [&](int s) { return bar0 + 8u * (2 * NPK + s); };
+  auto op_empty = [&](int s) { return bar0 + 8u * (2 * NPK + NS + s); };
+  auto acc_full = [&](int b) { return bar0 + 8u * (2 * NPK + 2 * NS + b); };
+  auto acc_empty = [&](int b) { return bar0 + 8u * (2 * NPK + 2 * NS + 2 + b); };
+  volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(smem + L::kMiscOff);
+  volatile uint32_t* abort_flag = misc + 1;
+  float* c_s = reinterpret_cast<float*>(smem + L::kVecOff);        // act_scale * post[t]
+  float* rs_s = c_s + kMaxTok;                                      // residual scale per token
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int nctas = gridDim.x;
+  const long long g_begin = range_start(D, blockIdx.x, nctas);
+  const long long g_end = range_start(D, blockIdx.x + 1, nctas);
+  const uint32_t pkx_bytes = (uint32_t)D.npad * PK_ROW;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < NPK; ++s) { mbar_init(pk_full(s), 1); mbar_init(pk_empty(s), 6); }
+    for (int s = 0; s < NS; ++s) { mbar_init(op_full(s), 6); mbar_init(op_empty(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 4); }
+    misc[1] = 0;
+    fence_mbar_init();
+    prefetch_tmap(&tmW);
+    prefetch_tmap(&tmX);
+  }
+  if (threadIdx.x >= kEpiWarp0 * 32 && threadIdx.x < kEpiWarp0 * 32 + kMaxTok) {
+    const int t = threadIdx.x - kEpiWarp0 * 32;
+    c_s[t] = (t < P.M && P.post) ? __fmul_rn(P.act_scale, __ldg(P.post + t)) : P.act_scale;
+    rs_s[t] = (t < P.M && P.res_scale) ? __ldg(P.res_scale + t) : 1.0f;
+  }
+  if (warp == 1) {
+    tmem_alloc(sbase + L::kMiscOff, kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = misc[0];
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int s = 0; uint32_t ph = 0;
+      uint32_t armed = 0, armed_par = 0;
+      bool ok = true;
+      for (long long g = g_begin; g < g_end; ++g) {
+        const int tile = (int)(g / D.kblocks), kb = (int)(g % D.kblocks);
+        if (!mbar_wait(pk_empty(s), ph ^ 1u, abort_flag, P.status, 1)) { ok = false; break; }
+        mbar_arrive_expect_tx(pk_full(s), L::kPkW + pkx_bytes);
+        tma_load_2d(sbase + L::kPkWOff + s * L::kPkW, &tmW, pk_full(s), kb * PK_ROW, tile * HR);
+        tma_load_2d(sbase + L::kPkXOff + s * L::kPkX, &tmX, pk_full(s), kb * PK_ROW, 0);
+        armed |= 1u << s;
+        armed_par = (armed_par & ~(1u << s)) | (ph << s);
+        if (++s == NPK) { s = 0; ph ^= 1u; }
+      }
+      if (!ok) {
+        const uint64_t t0 = globaltimer_ns();
+        for (int q = 0; q < NPK; ++q)
+          if (armed & (1u << q))
+            while (!mbar_try_wait(pk_full(q), (armed_par >> q) & 1u) && globaltimer_ns() - t0 < 2000000ull) {}
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc_i8(HR, D.npad, true, !P.a_unsigned);
+      int s = 0; uint32_t ph = 0; int seg = 0;
+      long long g = g_begin;
+      bool ok = true;
+      while (ok && g < g_end) {
+        const int kb0 = (int)(g % D.kblocks);
+        const long long left = g_end - g;
+        const int kb1 = (D.kblocks - kb0) < left ? D.kblocks : kb0 + (int)left;
+        const int b = seg & 1; const uint32_t bph = (seg >> 1) & 1;
+        if (!mbar_wait(acc_empty(b), bph ^ 1u, abort_flag, P.status, 2)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + b * kAccCols;
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!mbar_wait(op_full(s), ph, abort_flag, P.status, 3)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t bdesc = umma_desc_kmajor_sw128(sbase + L::kB8Off + s * L::kB8Stage);
+          const uint32_t a_tmem = tmem_base + kAStage0 + s * 32;
+#pragma unroll
+          for (int kk = 0; kk < BK / 32; ++kk)
+            umma_i8_ts(d_tmem, a_tmem + 8u * kk, bdesc + 2u * kk, idesc, (kb != kb0) || kk != 0);
+          umma_commit(op_empty(s));
+          if (++s == NS) { s = 0; ph ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit(acc_full(b));
+        g += kb1 - kb0;
+        ++seg;
+      }
+    }
+  } else if (warp < kConvAWarp0) {
+    // ------------------------------------------------------------------ token converters -> shared int8 tile
+    const int ctid = threadIdx.x - kConvBWarp0 * 32;     // 0..63
+    const int per_thread = D.npad / 16;                  // 16-byte chunks per thread: npad * 4 / 64
+    int ps = 0, s = 0; uint32_t pph = 0, ph = 0;
+    for (long long g = g_begin; g < g_end; ++g) {
+      if (!mbar_wait(pk_full(ps), pph, abort_flag, P.status, 7)) break;
+      const uint4* src = reinterpret_cast<const uint4*>(smem + L::kPkXOff + ps * L::kPkX);
+      uint4 c[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) if (i < per_thread) c[i] = src[i * 64 + ctid];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(pk_empty(ps));
+      if (!mbar_wait(op_empty(s), ph ^ 1u, abort_flag, P.status, 8)) break;
+      uint8_t* dst = smem + L::kB8Off + s * L::kB8Stage;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        if (i < per_thread) {
+          const int id = i * 64 + ctid;                  // 16-byte packed chunk: row id/4, chunk id%4
+          const int r = id >> 2, ch = id & 3;
+          uint32_t w[8];
+          widen(c[i], w);
+          uint8_t* rowp = dst + r * I8_ROW;
+          *reinterpret_cast<uint4*>(rowp + (((2 * ch) ^ (r & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(rowp + (((2 * ch + 1) ^ (r & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+        }
+      }
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(op_full(s));
+      if (++ps == NPK) { ps = 0; pph ^= 1u; }
+      if (++s == NS) { s = 0; ph ^= 1u; }
+    }
+  } else if (warp < kEpiWarp0) {
+    // ------------------------------------------------------------------ weight converters -> tensor memory
+    const int quad = warp & 3;                           // TMEM lanes this warp may touch
+    const int grp = (warp - kConvAWarp0) >> 2;           // takes the k-blocks whose running index has this parity
+    const int r = quad * 32 + lane;
+    const uint32_t swz = (uint32_t)((r >> 1) & 3);       // SWIZZLE_64B of the packed weight tile
+    long long kc = grp;                                  // running k-block index of this CTA
+    for (long long g = g_begin + grp; g < g_end; g += 2, kc += 2) {
+      const int ps = (int)(kc % NPK); const uint32_t pph = (uint32_t)((kc / NPK) & 1);
+      const int s = (int)(kc % NS);   const uint32_t ph = (uint32_t)((kc / NS) & 1);
+      if (!mbar_wait(pk_full(ps), pph, abort_flag, P.status, 5)) break;
+      const uint8_t* src = smem + L::kPkWOff + ps * L::kPkW + r * PK_ROW;
+      uint4 c[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) c[j] = *reinterpret_cast<const uint4*>(src + (((uint32_t)j ^ swz) << 4));
+      uint32_t v[32];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) widen(c[j], v + 8 * j);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(pk_empty(ps));
+      if (!mbar_wait(op_empty(s), ph ^ 1u, abort_flag, P.status, 6)) break;
+      tc_fence_after();
+      tmem_st_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + kAStage0 + s * 32, v);
+      tmem_wait_st();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(op_full(s));
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue
+    const int quad = warp & 3;
+    const int npad = D.npad;
+    int seg = 0;
+    long long g = g_begin;
+    while (g < g_end) {
+      const int tile = (int)(g / D.kblocks), kb0 = (int)(g % D.kblocks);
+      const long long left = g_end - g;
+      const int kb1 = (D.kblocks - kb0) < left ? D.kblocks : kb0 + (int)left;
+      const bool whole = kb0 == 0 && kb1 == D.kblocks;
+      const int b = seg & 1; const uint32_t bph = (seg >> 1) & 1;
+      const int n = tile * HR + quad * 32 + lane;        // weight row = output feature of this thread
+      const bool n_ok = n < P.N;
+      // per-row constants, fetched while the matmul of the segment runs
+      const float swn = n_ok ? load_scale(P.sw, P.scale_dtype, n) : 0.0f;
+      const int zw = (P.wsum && n_ok) ? P.zero_point * __ldg(P.wsum + n) : 0;
+      if (!mbar_wait(acc_full(b), bph, abort_flag, P.status, 4)) break;
+      tc_fence_after();
+      uint32_t v[kMaxTok];
+      const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + b * kAccCols;
+      {
+        uint32_t t16[16];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          if (q * 16 < npad) {
+            tmem_ld_32x16(taddr + q * 16, t16);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[q * 16 + j] = t16[j];
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty(b));
+
+      bool finalize = whole;
+      if (!whole) {
+        // raw partial sums -> this CTA's slot; the last contributor of the tile adds all slots up
+        const int my_slot = (g == g_begin) ? 0 : 1;
+        int32_t* slot = D.slots + ((size_t)(blockIdx.x * 2 + my_slot) * npad) * HR + quad * 32 + lane;
+#pragma unroll
+        for (int t = 0; t < kMaxTok; ++t) if (t < npad) slot[(size_t)t * HR] = (int32_t)v[t];
+        __threadfence();
+        __syncwarp();
+        // contributors of this tile: every CTA whose range meets [tile*KB, (tile+1)*KB)
+        const long long t_begin = (long long)tile * D.kblocks, t_end = t_begin + D.kblocks;
+        int c_first = blockIdx.x, c_last = blockIdx.x;
+        while (c_first > 0 && range_start(D, c_first, nctas) > t_begin) --c_first;
+        while (c_last + 1 < nctas && range_start(D, c_last + 1, nctas) < t_end) ++c_last;
+        const uint32_t expected = (uint32_t)(c_last - c_first + 1);
+        uint32_t old = 0;
+        if (lane == 0) old = atomicAdd(D.counters + tile * 4 + quad, 1u);
+        old = __shfl_sync(0xffffffffu, old, 0);
+        if (old == expected - 1) {
+          __threadfence();
+#pragma unroll
+          for (int t = 0; t < kMaxTok; ++t) v[t] = 0;
+          for (int c = c_first; c <= c_last; ++c) {
+            const int cs = (range_start(D, c, nctas) >= t_begin) ? 0 : 1;
+            const int32_t* src = D.slots + ((size_t)(c * 2 + cs) * npad) * HR + quad * 32 + lane;
+#pragma unroll
+            for (int t = 0; t < kMaxTok; ++t) if (t < npad) v[t] += (uint32_t)__ldcg(src + (size_t)t * HR);
+          }
+          if (lane == 0) D.counters[tile * 4 + quad] = 0;      // ready for the next launch
+          finalize = true;
+        }
+      }
+      if (finalize && n_ok) {
+#pragma unroll
+        for (int t = 0; t < kMaxTok; ++t) {
+          if (t < P.M) {
+            const int a = (((int)v[t]) >> 8) - zw;
+            if (P.acc_out) P.acc_out[(size_t)t * P.N + n] = a;
+            if (P.Y) {
+              float y = __fmul_rn(__fmul_rn((float)a, swn), c_s[t]);
+              if (P.residual)
+                y = __fadd_rn(y, __fmul_rn(__bfloat162float(P.residual[(size_t)t * P.N + n]), rs_s[t]));
+              P.Y[(size_t)t * P.N + n] = __float2bfloat16_rn(y);
+            }
+          }
+        }
+      }
+      g += kb1 - kb0;
+      ++seg;
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+static bool make_map(CUtensorMap* m, const void* base, int rows, int K, int box_rows, CUtensorMapSwizzle swz) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)(K / 2), (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)(K / 2)};
+  const cuuint32_t box[2] = {(cuuint32_t)PK_ROW, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static int num_sms() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (n <= 0) n = 1;
+  }
+  return n;
+}
+
+}  // namespace decode
+
+int decode_npad(int M) { return M <= 16 ? 16 : M <= 32 ? 32 : 64; }
+
+size_t gemm_decode_scratch_bytes(int M) {
+  return (size_t)kDecodeMaxCtas * 2 * (size_t)decode_npad(M) * decode::HR * sizeof(int32_t);
+}
+
+// Xq [M <= 64, K/2], Wq [N, K/2]; `scratch` holds gemm_decode_scratch_bytes(M) bytes; the counters
+// live in the workspace's control block behind the status word.
+int gemm_decode_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, const GemmParams& P, void* scratch) {
+  using namespace decode;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(gemm_w4a4_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::kAlloc) !=
+        cudaSuccess)
+      return FPT_ERR_CUDA;
+    attr_set = true;
+  }
+  DecodeParams D;
+  D.g = P;
+  D.npad = decode_npad(P.M);
+  D.tiles = (P.N + HR - 1) / HR;
+  D.kblocks = P.K / BK;
+  D.total = (long long)D.tiles * D.kblocks;
+  D.whole_tiles = D.tiles * 4 > kDecodeMaxCounters ? 1 : 0;
+  D.slots = reinterpret_cast<int32_t*>(scratch);
+  D.counters = P.status + kCounterWord0;
+  CUtensorMap tmW, tmX;
+  if (!make_map(&tmW, Wq, P.N, P.K, HR, CU_TENSOR_MAP_SWIZZLE_64B) ||
+      !make_map(&tmX, Xq, P.M, P.K, D.npad, CU_TENSOR_MAP_SWIZZLE_NONE))
+    return FPT_ERR_CUDA;
+  int ctas = num_sms() < kDecodeMaxCtas ? num_sms() : kDecodeMaxCtas;
+  const long long units = D.whole_tiles ? D.tiles : D.total;
+  if (units < ctas) ctas = (int)units;
+  gemm_w4a4_decode_kernel<<<ctas, kThreads, Smem::kAlloc, st>>>(tmW, tmX, D);
+  return cudaGetLastError() == cudaSuccess ? FPT_OK : FPT_ERR_CUDA;
+}
+
+}  // namespace fpt

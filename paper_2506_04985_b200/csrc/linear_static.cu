@@ -62,18 +62,20 @@ extern "C" int fpt_w4a4_linear_static(void* stream, const void* X, int M, int K,
   if (post_mode == FPT_POST_VECTOR && !post) return FPT_ERR_BAD_ARG;
   if (scale_dtype != FPT_DTYPE_F32 && scale_dtype != FPT_DTYPE_F16) return FPT_ERR_BAD_ARG;
   if (((uintptr_t)X | (uintptr_t)Wq | (uintptr_t)Y) & 15) return FPT_ERR_ALIGNMENT;
-  // status block | packed codes [M, K/2] | one float per token
+  // control block | matmul scratch (decode sizes only) | packed codes [M, K/2] | one float per token
   const size_t codes = up256s((size_t)M * (size_t)K / 2);
-  const size_t need = kStatusBytes + codes + up256s((size_t)M * 4);
+  const size_t gemm_ws = kStatusBytes + gemm_scratch_bytes(M);
+  const size_t need = gemm_ws + codes + up256s((size_t)M * 4);
   if (need > kStaticScratchBytes) return FPT_ERR_WORKSPACE;     // the built-in scratch is too small for M x K
 
   unsigned char* base = nullptr;
   int rc = static_scratch(&base);
   if (rc) return rc;
   cudaStream_t st = (cudaStream_t)stream;
-  // the array keeps whatever the last call left: the status word has to start at zero
+  // the array keeps whatever the last call left: the control block (status word, tile counters)
+  // has to start at zero
   if (cudaMemsetAsync(base, 0, kStatusBytes, st) != cudaSuccess) return FPT_ERR_CUDA;
-  uint8_t* Xq = base + kStatusBytes;
+  uint8_t* Xq = base + gemm_ws;
   float* post_inv = reinterpret_cast<float*>(Xq + codes);
   if (act_quant_launch(st, X, M, K, K, act_qp, flags, eps, nullptr, s_in, Xq, s_out,
                        post_mode == FPT_POST_INVERSE_OF_PRE ? post_inv : nullptr, nullptr) != cudaSuccess)
@@ -89,5 +91,6 @@ extern "C" int fpt_w4a4_linear_static(void* stream, const void* X, int M, int K,
   P.post = pv;
   P.Y = reinterpret_cast<__nv_bfloat16*>(Y);
   P.status = reinterpret_cast<uint32_t*>(base);
+  P.scratch = base + kStatusBytes;
   return gemm_launch(st, Xq, Wq, P);
 }

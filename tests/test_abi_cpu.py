@@ -36,7 +36,8 @@ def test_version_and_strerror(B):
 
 
 def test_workspace_sizes(B):
-    assert B.fpt_workspace_bytes(B.OP_GEMM, 128, 1024, 1024) >= 256
+    assert B.fpt_workspace_bytes(B.OP_GEMM, 128, 1024, 1024) >= 8192
+    assert B.fpt_workspace_bytes(B.OP_GEMM, 64, 1024, 1024) > B.fpt_workspace_bytes(B.OP_GEMM, 128, 1024, 1024)
     lin = B.fpt_workspace_bytes(B.OP_LINEAR, 2048, 4096, 4096)
     assert lin >= 2048 * 4096 // 2 + 2048 * 4
     mlp = B.fpt_workspace_bytes(B.OP_MLP, 4096, 14336, 4096)
@@ -67,14 +68,14 @@ def test_argument_errors_are_reported_before_any_launch(B):
     # matmul: K must be a multiple of 128, N of 8, workspace present and large enough
     args = lambda M, N, K, ws, wsb: (None, fake, fake, M, N, K, fake, B.DTYPE_F32, None, 0.5, 1, 0, None, None, None,
                                      fake, None, ws, wsb)
-    assert L.fpt_w4a4_gemm(*args(16, 64, 96, fake, 256)) == B.ERR_UNSUPPORTED
-    assert L.fpt_w4a4_gemm(*args(16, 60, 128, fake, 256)) == B.ERR_UNSUPPORTED
+    assert L.fpt_w4a4_gemm(*args(16, 64, 96, fake, 1 << 30)) == B.ERR_UNSUPPORTED
+    assert L.fpt_w4a4_gemm(*args(16, 60, 128, fake, 1 << 30)) == B.ERR_UNSUPPORTED
     assert L.fpt_w4a4_gemm(*args(16, 64, 128, None, 0)) == B.ERR_WORKSPACE
     assert L.fpt_w4a4_gemm(*args(16, 64, 128, fake, 8)) == B.ERR_WORKSPACE
-    assert L.fpt_w4a4_gemm(*args(0, 64, 128, fake, 256)) == B.ERR_BAD_ARG
+    assert L.fpt_w4a4_gemm(*args(0, 64, 128, fake, 1 << 30)) == B.ERR_BAD_ARG
     # asymmetric activations need the weight row sums
     r = L.fpt_w4a4_gemm(None, fake, fake, 16, 64, 128, fake, B.DTYPE_F32, None, 0.5, 0, 8, None, None, None, fake,
-                        None, fake, 256)
+                        None, fake, 1 << 30)
     assert r == B.ERR_BAD_ARG
     r = L.fpt_quantize_weights(None, fake, B.DTYPE_BF16, 8, 128, ctypes.byref(B.QParams(4, False, 1.0, 8)),
                                B.RANGE_MINMAX, 3.0, B.DTYPE_F32, fake, fake, None)

@@ -40,7 +40,7 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point():
 
 def test_size_beyond_the_built_in_scratch_is_refused_before_any_launch():
     M, K, N = 8192, 8192, 8          # 32 MiB of codes: more than the array holds
-    assert 256 + M * K // 2 > B.STATIC_SCRATCH_BYTES
+    assert B.fpt_workspace_bytes(B.OP_LINEAR, M, N, K) > B.STATIC_SCRATCH_BYTES
     x = torch.zeros((M, K), dtype=torch.bfloat16, device="cuda")
     wq = torch.zeros((N, K // 2), dtype=torch.uint8, device="cuda")
     sw = torch.ones((N,), dtype=torch.float32, device="cuda")
