@@ -8,7 +8,7 @@
 // (tcgen05.st), the MMA reads them from there; only the few token rows are widened into a
 // shared-memory tile.  Nothing of the weight stream is ever stored to shared memory twice.
 //
-// Work is split stream-K style: the T = (N/128) * (K/128) weight k-blocks are cut into equal
+// Work is split stream-K style: the T = (N/128) * (K/256) weight k-blocks are cut into equal
 // contiguous ranges, one per CTA (one CTA per SM), so every SM streams the same number of bytes
 // whatever the shape.  A range that covers part of a tile leaves its raw int32 partial sums in
 // a scratch slot; the last CTA to arrive at a tile (an atomic counter per tile and lane
@@ -26,11 +26,11 @@ namespace fpt {
 namespace decode {
 
 constexpr int HR = 128;                    // weight rows per tile
-constexpr int BK = 128;                    // codes per k-block
+constexpr int BK = 256;                    // codes per k-block: 128 packed bytes per row, one full cache line
 constexpr int PK_ROW = BK / 2;
-constexpr int I8_ROW = BK;
-constexpr int NS = 8;                      // widened stages: 8 x 32 tensor-memory columns + 8 token tiles
-constexpr int NPK = 12;                    // packed stages in flight from TMA
+constexpr int I8_ROW = 128;                // the widened token tile is two 128-byte-swizzled halves of 128 codes
+constexpr int NS = 4;                      // widened stages: 4 x 64 tensor-memory columns + 4 token tiles
+constexpr int NPK = 6;                     // packed stages in flight from TMA
 constexpr int kMaxTok = 64;
 constexpr int kAccCols = 64;               // per accumulator buffer (two of them)
 constexpr int kAStage0 = 2 * kAccCols;
@@ -39,9 +39,10 @@ constexpr int kThreads = 512;
 constexpr int kConvBWarp0 = 2, kConvAWarp0 = 4, kEpiWarp0 = 12;
 
 struct Smem {
-  static constexpr int kB8Stage = kMaxTok * I8_ROW;                 // 8 KB: widened token tile
-  static constexpr int kPkW = HR * PK_ROW;                          // 8 KB: packed weights of one k-block
-  static constexpr int kPkX = kMaxTok * PK_ROW;                     // 4 KB: packed tokens of one k-block
+  static constexpr int kB8Half = kMaxTok * I8_ROW;                  // 8 KB: 64 token rows x 128 codes as int8
+  static constexpr int kB8Stage = 2 * kB8Half;                      // 16 KB: widened token tile
+  static constexpr int kPkW = HR * PK_ROW;                          // 16 KB: packed weights of one k-block
+  static constexpr int kPkX = kMaxTok * PK_ROW;                     // 8 KB: packed tokens of one k-block
   static constexpr int kB8Off = 0;
   static constexpr int kPkWOff = kB8Off + NS * kB8Stage;
   static constexpr int kPkXOff = kPkWOff + NPK * kPkW;
@@ -58,7 +59,7 @@ struct DecodeParams {
   GemmParams g;            // M = tokens, N = weight rows, K
   int npad;                // tokens padded to the MMA N: 16, 32 or 64
   int tiles;               // N / 128 rounded up
-  int kblocks;             // K / 128
+  int kblocks;             // K / 256 rounded up (a half block at the end reads zeros past the row)
   long long total;         // tiles * kblocks
   int whole_tiles;         // 1: ranges end on tile boundaries (no partial sums, no counters)
   int32_t* slots;          // [gridDim.x][2][npad][128] raw int32 partial sums
@@ -169,11 +170,12 @@ gemm_w4a4_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(op_full(s), ph, abort_flag, P.status, 3)) { ok = false; break; }
           tc_fence_after();
-          const uint64_t bdesc = umma_desc_kmajor_sw128(sbase + L::kB8Off + s * L::kB8Stage);
-          const uint32_t a_tmem = tmem_base + kAStage0 + s * 32;
+          const uint32_t a_tmem = tmem_base + kAStage0 + s * (BK / 4);
 #pragma unroll
-          for (int kk = 0; kk < BK / 32; ++kk)
-            umma_i8_ts(d_tmem, a_tmem + 8u * kk, bdesc + 2u * kk, idesc, (kb != kb0) || kk != 0);
+          for (int kk = 0; kk < BK / 32; ++kk) {
+            const uint64_t bdesc = umma_desc_kmajor_sw128(sbase + L::kB8Off + s * L::kB8Stage + (kk >> 2) * L::kB8Half);
+            umma_i8_ts(d_tmem, a_tmem + 8u * kk, bdesc + 2u * (kk & 3), idesc, (kb != kb0) || kk != 0);
+          }
           umma_commit(op_empty(s));
           if (++s == NS) { s = 0; ph ^= 1u; }
         }
@@ -186,26 +188,26 @@ gemm_w4a4_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
   } else if (warp < kConvAWarp0) {
     // ------------------------------------------------------------------ token converters -> shared int8 tile
     const int ctid = threadIdx.x - kConvBWarp0 * 32;     // 0..63
-    const int per_thread = D.npad / 16;                  // 16-byte chunks per thread: npad * 4 / 64
+    const int per_thread = D.npad / 8;                   // 16-byte chunks per thread: npad * 8 / 64
     int ps = 0, s = 0; uint32_t pph = 0, ph = 0;
     for (long long g = g_begin; g < g_end; ++g) {
       if (!mbar_wait(pk_full(ps), pph, abort_flag, P.status, 7)) break;
       const uint4* src = reinterpret_cast<const uint4*>(smem + L::kPkXOff + ps * L::kPkX);
-      uint4 c[4];
+      uint4 c[8];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) if (i < per_thread) c[i] = src[i * 64 + ctid];
+      for (int i = 0; i < 8; ++i) if (i < per_thread) c[i] = src[i * 64 + ctid];
       __syncwarp();
       if (lane == 0) mbar_arrive(pk_empty(ps));
       if (!mbar_wait(op_empty(s), ph ^ 1u, abort_flag, P.status, 8)) break;
       uint8_t* dst = smem + L::kB8Off + s * L::kB8Stage;
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
+      for (int i = 0; i < 8; ++i) {
         if (i < per_thread) {
-          const int id = i * 64 + ctid;                  // 16-byte packed chunk: row id/4, chunk id%4
-          const int r = id >> 2, ch = id & 3;
+          const int id = i * 64 + ctid;                  // 16-byte packed chunk: row id/8, chunk id%8
+          const int r = id >> 3, ch = id & 3;            // chunks 0-3: first 128 codes, 4-7: second half
           uint32_t w[8];
           widen(c[i], w);
-          uint8_t* rowp = dst + r * I8_ROW;
+          uint8_t* rowp = dst + ((id >> 2) & 1) * L::kB8Half + r * I8_ROW;
           *reinterpret_cast<uint4*>(rowp + (((2 * ch) ^ (r & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
           *reinterpret_cast<uint4*>(rowp + (((2 * ch + 1) ^ (r & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
         }
@@ -221,24 +223,26 @@ gemm_w4a4_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     const int quad = warp & 3;                           // TMEM lanes this warp may touch
     const int grp = (warp - kConvAWarp0) >> 2;           // takes the k-blocks whose running index has this parity
     const int r = quad * 32 + lane;
-    const uint32_t swz = (uint32_t)((r >> 1) & 3);       // SWIZZLE_64B of the packed weight tile
+    const uint32_t swz = (uint32_t)(r & 7);              // SWIZZLE_128B of the packed weight tile
     long long kc = grp;                                  // running k-block index of this CTA
     for (long long g = g_begin + grp; g < g_end; g += 2, kc += 2) {
       const int ps = (int)(kc % NPK); const uint32_t pph = (uint32_t)((kc / NPK) & 1);
       const int s = (int)(kc % NS);   const uint32_t ph = (uint32_t)((kc / NS) & 1);
       if (!mbar_wait(pk_full(ps), pph, abort_flag, P.status, 5)) break;
       const uint8_t* src = smem + L::kPkWOff + ps * L::kPkW + r * PK_ROW;
-      uint4 c[4];
+      uint4 c[8];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) c[j] = *reinterpret_cast<const uint4*>(src + (((uint32_t)j ^ swz) << 4));
-      uint32_t v[32];
+      for (int j = 0; j < 8; ++j) c[j] = *reinterpret_cast<const uint4*>(src + (((uint32_t)j ^ swz) << 4));
+      uint32_t v[64];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) widen(c[j], v + 8 * j);
+      for (int j = 0; j < 8; ++j) widen(c[j], v + 8 * j);
       __syncwarp();
       if (lane == 0) mbar_arrive(pk_empty(ps));
       if (!mbar_wait(op_empty(s), ph ^ 1u, abort_flag, P.status, 6)) break;
       tc_fence_after();
-      tmem_st_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + kAStage0 + s * 32, v);
+      const uint32_t a_tmem = tmem_base + ((uint32_t)(quad * 32) << 16) + kAStage0 + s * (BK / 4);
+      tmem_st_32x32(a_tmem, v);
+      tmem_st_32x32(a_tmem + 32, v + 32);
       tmem_wait_st();
       tc_fence_before();
       __syncwarp();
@@ -303,11 +307,28 @@ gemm_w4a4_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
           __threadfence();
 #pragma unroll
           for (int t = 0; t < kMaxTok; ++t) v[t] = 0;
-          for (int c = c_first; c <= c_last; ++c) {
-            const int cs = (range_start(D, c, nctas) >= t_begin) ? 0 : 1;
-            const int32_t* src = D.slots + ((size_t)(c * 2 + cs) * npad) * HR + quad * 32 + lane;
+          if (npad == 16) {
+            // few values per contributor: keep the loads of four contributors in flight together
+            for (int c = c_first; c <= c_last; c += 4) {
+              uint32_t w[4][16];
 #pragma unroll
-            for (int t = 0; t < kMaxTok; ++t) if (t < npad) v[t] += (uint32_t)__ldcg(src + (size_t)t * HR);
+              for (int u = 0; u < 4; ++u) {
+                const int cc = c + u <= c_last ? c + u : c_last;
+                const int cs = (range_start(D, cc, nctas) >= t_begin) ? 0 : 1;
+                const int32_t* src = D.slots + ((size_t)(cc * 2 + cs) * npad) * HR + quad * 32 + lane;
+#pragma unroll
+                for (int t = 0; t < 16; ++t) w[u][t] = (c + u <= c_last) ? (uint32_t)__ldcg(src + (size_t)t * HR) : 0u;
+              }
+#pragma unroll
+              for (int t = 0; t < 16; ++t) v[t] += (w[0][t] + w[1][t]) + (w[2][t] + w[3][t]);
+            }
+          } else {
+            for (int c = c_first; c <= c_last; ++c) {
+              const int cs = (range_start(D, c, nctas) >= t_begin) ? 0 : 1;
+              const int32_t* src = D.slots + ((size_t)(c * 2 + cs) * npad) * HR + quad * 32 + lane;
+#pragma unroll
+              for (int t = 0; t < kMaxTok; ++t) if (t < npad) v[t] += (uint32_t)__ldcg(src + (size_t)t * HR);
+            }
           }
           if (lane == 0) D.counters[tile * 4 + quad] = 0;      // ready for the next launch
           finalize = true;
@@ -408,16 +429,26 @@ int gemm_decode_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, co
   D.g = P;
   D.npad = decode_npad(P.M);
   D.tiles = (P.N + HR - 1) / HR;
-  D.kblocks = P.K / BK;
+  D.kblocks = (P.K + BK - 1) / BK;
   D.total = (long long)D.tiles * D.kblocks;
   D.whole_tiles = D.tiles * 4 > kDecodeMaxCounters ? 1 : 0;
   D.slots = reinterpret_cast<int32_t*>(scratch);
   D.counters = P.status + kCounterWord0;
   CUtensorMap tmW, tmX;
-  if (!make_map(&tmW, Wq, P.N, P.K, HR, CU_TENSOR_MAP_SWIZZLE_64B) ||
+  if (!make_map(&tmW, Wq, P.N, P.K, HR, CU_TENSOR_MAP_SWIZZLE_128B) ||
       !make_map(&tmX, Xq, P.M, P.K, D.npad, CU_TENSOR_MAP_SWIZZLE_NONE))
     return FPT_ERR_CUDA;
-  int ctas = num_sms() < kDecodeMaxCtas ? num_sms() : kDecodeMaxCtas;
+  // Number of CTAs (= equal ranges of the weight stream).  With fewer tiles than SMs each tile is
+  // cut into the same number of ranges, so that range ends fall on tile ends (fewest partial sums);
+  // with more tiles than SMs every SM gets the same share and ranges end where they end.
+  const int sms = num_sms() < kDecodeMaxCtas ? num_sms() : kDecodeMaxCtas;
+  int ctas = sms;
+  if (D.tiles <= sms) {
+    int split = sms / D.tiles;
+    const int max_split = D.kblocks / 2 > 0 ? D.kblocks / 2 : 1;      // at least 2 k-blocks (512 codes) per range
+    if (split > max_split) split = max_split;
+    ctas = D.tiles * split;
+  }
   const long long units = D.whole_tiles ? D.tiles : D.total;
   if (units < ctas) ctas = (int)units;
   gemm_w4a4_decode_kernel<<<ctas, kThreads, Smem::kAlloc, st>>>(tmW, tmX, D);

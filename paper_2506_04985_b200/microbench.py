@@ -9,7 +9,8 @@
 Operands are random packed codes / random bf16 values made on the device (timing does
 not depend on the values).  `--sets S` rotates S independent operand sets so that every
 launch reads HBM rather than the L2 (pick S so that S x bytes-per-set exceeds 126 MB);
-`--reps R` launches are timed back to back between two events on the launching stream.
+`--reps R` launches are timed back to back between two events on the launching stream
+(`--graph`: captured once in a CUDA graph and replayed, for kernels shorter than a launch).
 Prints one JSON line: microseconds per launch, TOP/s, GB/s of algorithmic bytes.
 The same command with small `--reps` is what the profiler captures.
 """
@@ -94,6 +95,27 @@ def time_case(runs, reps, warmup=3):
     return e0.elapsed_time(e1) * 1e3 / reps
 
 
+def time_case_graph(runs, reps, warmup=3, replays=5):
+    """The same `reps` launches captured once in a CUDA graph and replayed: removes the host's
+    launch cost (argument marshalling, tensor-map encoding) from kernels of a few microseconds."""
+    for i in range(max(warmup, 1)):
+        runs[i % len(runs)]()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for i in range(reps):
+            runs[i % len(runs)]()
+    g.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(replays):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) * 1e3 / (reps * replays)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("kind", choices=["gemm", "act_quant", "silu_quant", "linear", "mlp"])
@@ -104,12 +126,13 @@ def main():
     ap.add_argument("--reps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--f16-scales", action="store_true")
+    ap.add_argument("--graph", action="store_true", help="replay the launches from a CUDA graph")
     a = ap.parse_args()
     B.lib()
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
     runs, ops, nbytes = make_case(a.kind, a.M, a.N, a.K, a.sets, dev, a.f16_scales)
-    us = time_case(runs, a.reps, a.warmup)
+    us = time_case_graph(runs, a.reps, a.warmup) if a.graph else time_case(runs, a.reps, a.warmup)
     print(json.dumps({"kind": a.kind, "M": a.M, "N": a.N, "K": a.K, "sets": a.sets, "reps": a.reps,
                       "us": us, "tops": ops / us / 1e6, "gbs": nbytes / us / 1e3}))
 
