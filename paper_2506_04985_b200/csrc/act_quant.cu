@@ -19,8 +19,8 @@ struct ActQuantParams {
   int flags;
   float eps;
   float inv_delta;     // 1 / D, rounded once on the host
-  float lo, hi;        // qmin - z, qmax - z
-  float magic;         // 1.5 * 2^23 + z
+  int   qmax_minus_z;  // upper end of the grid minus the zero point
+  uint32_t flip;       // see quant_word
 };
 
 // 2^f on [-0.5, 0.5]: degree-6 Taylor coefficients (ln 2)^k / k!, rounded to float32.
@@ -51,31 +51,95 @@ __device__ __forceinline__ uint32_t silu_mul_pair(uint32_t g, uint32_t u) {
   return f32_to_bf16_bits(lo) | (f32_to_bf16_bits(hi) << 16);
 }
 
-__device__ __forceinline__ uint32_t quant_nibble(float x, float p, const ActQuantParams& P) {
-  float u = __fmul_rn(__fmul_rn(x, p), P.inv_delta);
-  u = fminf(fmaxf(u, P.lo), P.hi);                           // NaN -> lo
-  return __float_as_uint(__fadd_rn(u, P.magic)) & 0xFu;      // rne(u) + z in the low mantissa bits
+// Two float32 lanes in one 64-bit register: sm_100 multiplies both with one instruction, each
+// lane rounded to nearest even on its own (the same result as two scalar multiplies).
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t mul_f32x2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
 }
 
-__device__ __forceinline__ uint32_t quant_word(const uint4& v, float p, const ActQuantParams& P) {
-  uint32_t w;
-  w  = quant_nibble(bf16lo_to_f32(v.x), p, P);
-  w |= quant_nibble(bf16hi_to_f32(v.x), p, P) << 4;
-  w |= quant_nibble(bf16lo_to_f32(v.y), p, P) << 8;
-  w |= quant_nibble(bf16hi_to_f32(v.y), p, P) << 12;
-  w |= quant_nibble(bf16lo_to_f32(v.z), p, P) << 16;
-  w |= quant_nibble(bf16hi_to_f32(v.z), p, P) << 20;
-  w |= quant_nibble(bf16lo_to_f32(v.w), p, P) << 24;
-  w |= quant_nibble(bf16hi_to_f32(v.w), p, P) << 28;
-  return w;
+// Quantiser arithmetic of one 16-byte chunk (8 values), in the order the header states:
+//   u = (x * p) * (1/D)          two separately rounded float32 multiplies
+//   q = clamp(rne(u) + z)        a NaN maps to the lowest code
+// evaluated on the NEGATED value v = (x * -p) * (1/D) = -u (negation is exact and rounding to
+// nearest even is symmetric): adding 1.5 * 2^23 leaves -rne(u) in the low mantissa bits, and the
+// float's bit pattern is monotone in v, also beyond the exact range and for +Inf and NaN, which
+// are the largest patterns.  One integer add-min-relu then yields qmax - q in [0, 15] with the
+// NaN at qmax - qmin = 15, i.e. the lowest code; the nibbles are flipped back by one XOR per
+// word (15 - c = c ^ 15; on the symmetric grid the two's complement nibble of 7 - c is c ^ 7).
+struct QuantConsts {
+  uint64_t np2, d2, m2;   // (-p, -p), (1/D, 1/D), (magic, magic)
+  int bias;               // -(bits of magic) + (qmax - z)
+  uint32_t flip;          // 0x77777777 symmetric, 0xFFFFFFFF asymmetric
+};
+
+__device__ __forceinline__ QuantConsts quant_consts(float p, const ActQuantParams& P) {
+  QuantConsts c;
+  c.np2 = pack_f32x2(-p, -p);
+  c.d2 = pack_f32x2(P.inv_delta, P.inv_delta);
+  c.m2 = pack_f32x2(12582912.0f, 12582912.0f);
+  c.bias = -0x4B400000 + P.qmax_minus_z;
+  c.flip = P.flip;
+  return c;
 }
 
+// Two values of one 32-bit word -> (15 - code) each, the second in front: returns c0 + 16 * c1 + 256 * prev.
+__device__ __forceinline__ uint32_t quant_pair(uint32_t w, const QuantConsts& c, uint32_t prev) {
+  float v0, v1;
+  unpack_f32x2(add_f32x2(mul_f32x2(mul_f32x2(pack_f32x2(bf16lo_to_f32(w), bf16hi_to_f32(w)), c.np2), c.d2), c.m2), v0, v1);
+  // (a negative sum -- u beyond 1.2e7 -- has a negative pattern; max(., 0) keeps the add below from wrapping)
+  const uint32_t c0 = (uint32_t)__viaddmin_s32_relu(max(__float_as_int(v0), 0), c.bias, 15);
+  const uint32_t c1 = (uint32_t)__viaddmin_s32_relu(max(__float_as_int(v1), 0), c.bias, 15);
+  return (prev * 16u + c1) * 16u + c0;
+}
+
+__device__ __forceinline__ uint32_t quant_word(const uint4& v, const QuantConsts& c) {
+  uint32_t w = quant_pair(v.w, c, 0u);
+  w = quant_pair(v.z, c, w);
+  w = quant_pair(v.y, c, w);
+  w = quant_pair(v.x, c, w);
+  return w ^ c.flip;
+}
+
+// acc + the 8 squares of a chunk in float64.  The bf16 magnitude bits, moved to the top of a
+// float64's high word, are the value times 2^-896 for every finite input (normal, subnormal or
+// zero alike); one exact multiply by 2^896 restores it, the square is exact in float64 and the
+// fused add rounds once.  Inf and NaN inputs come out as huge finite numbers here: the caller
+// recognises them by the overflowing float32 sum and redoes the row with sumsq_exact.
 __device__ __forceinline__ double sumsq(const uint4& v, double acc) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+  const double rebias = __hiloint2double(0x77F00000, 0);            // 2^896
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const double a = __hiloint2double((int)((w[i] & 0x7FFFu) << 13), 0) * rebias;
+    const double b = __hiloint2double((int)((w[i] >> 3) & 0x0FFFE000u), 0) * rebias;
+    acc = fma(a, a, acc);
+    acc = fma(b, b, acc);
+  }
+  return acc;
+}
+
+// The same sum by the definition (float32 square, widened, added): used for rows with Inf / NaN.
+__device__ __forceinline__ double sumsq_exact(const uint4& v, double acc) {
   const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const float a = bf16lo_to_f32(w[i]), b = bf16hi_to_f32(w[i]);
-    acc += (double)__fmul_rn(a, a);            // the square of a bf16 value is exact in float32
+    acc += (double)__fmul_rn(a, a);
     acc += (double)__fmul_rn(b, b);
   }
   return acc;
@@ -127,6 +191,24 @@ __global__ void __launch_bounds__(T) act_quant_kernel(const ActQuantParams P) {
       double s = 0.0;
 #pragma unroll
       for (int w = 0; w < T / 32; ++w) s += warp_part[w];
+      bcast = (float)s;
+    }
+    __syncthreads();
+    if (!(bcast <= 3.4028234e38f)) {               // Inf / NaN in the row (or a genuine overflow): by the definition
+      __syncthreads();
+      acc = 0.0;
+#pragma unroll
+      for (int i = 0; i < V; ++i)
+        if (i * T + tid < chunks) acc = sumsq_exact(v[i], acc);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+      if ((tid & 31) == 0) warp_part[tid >> 5] = acc;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      double s = 0.0;
+#pragma unroll
+      for (int w = 0; w < T / 32; ++w) s += warp_part[w];
       const float ss = (float)s;                                        // one rounding to float32
       const float ms = __fdiv_rn(ss, (float)P.K);
       const float rho = __fsqrt_rn(__fadd_rn(ms, P.eps));
@@ -144,11 +226,188 @@ __global__ void __launch_bounds__(T) act_quant_kernel(const ActQuantParams P) {
     if (P.r_out) P.r_out[t] = r;
   }
   uint32_t* out = P.Xq + (size_t)t * (size_t)chunks;
+  const QuantConsts qc = quant_consts(p, P);
 #pragma unroll
   for (int i = 0; i < V; ++i) {
     const int c = i * T + tid;
-    if (c < chunks) out[c] = quant_word(v[i], p, P);
+    if (c < chunks) out[c] = quant_word(v[i], qc);
   }
+}
+
+// One warp per token for rows of up to 256 * V elements: the row lives in registers, the
+// reduction is a warp shuffle, no shared memory and no block-wide barrier.  W warps per CTA.
+template <int V, int W>
+__global__ void __launch_bounds__(W * 32) act_quant_warp_kernel(const ActQuantParams P) {
+  const int lane = threadIdx.x & 31;
+  const int t = blockIdx.x * W + (threadIdx.x >> 5);
+  if (t >= P.M) return;
+  const int chunks = P.K >> 3;
+  const uint4* row = P.X + (size_t)t * (size_t)(P.ldx >> 3);
+  uint4 v[V];
+#pragma unroll
+  for (int i = 0; i < V; ++i) {
+    const int c = i * 32 + lane;
+    if (c < chunks) v[i] = __ldg(row + c);
+  }
+  float r = 1.0f;
+  if (P.flags & FPT_RMSNORM) {
+    double acc0 = 0.0, acc1 = 0.0;                 // two chains: the float64 adds are latency-bound otherwise
+#pragma unroll
+    for (int i = 0; i < V; ++i)
+      if (i * 32 + lane < chunks) { if (i & 1) acc1 = sumsq(v[i], acc1); else acc0 = sumsq(v[i], acc0); }
+    double acc = acc0 + acc1;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (!((float)acc <= 3.4028234e38f)) {          // Inf / NaN in the row (or a genuine overflow): by the definition
+      acc0 = 0.0;
+#pragma unroll
+      for (int i = 0; i < V; ++i)
+        if (i * 32 + lane < chunks) acc0 = sumsq_exact(v[i], acc0);
+      acc = acc0;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    }
+    const float ss = (float)acc;                   // one rounding to float32 (every lane holds the same sum)
+    const float ms = __fdiv_rn(ss, (float)P.K);
+    const float rho = __fsqrt_rn(__fadd_rn(ms, P.eps));
+    r = __fdiv_rn(1.0f, rho);
+  }
+  const float s = P.s_in ? __ldg(P.s_in + t) : 1.0f;
+  const float rs = P.s_in ? __fmul_rn(r, s) : r;
+  const float p = (P.flags & FPT_SCALE_INPUT) ? rs : r;
+  if (lane == 0) {
+    if (P.s_out) P.s_out[t] = rs;
+    if (P.post_inv) P.post_inv[t] = __fdiv_rn(1.0f, p);
+    if (P.r_out) P.r_out[t] = r;
+  }
+  uint32_t* out = P.Xq + (size_t)t * (size_t)chunks;
+  const QuantConsts qc = quant_consts(p, P);
+#pragma unroll
+  for (int i = 0; i < V; ++i) {
+    const int c = i * 32 + lane;
+    if (c < chunks) out[c] = quant_word(v[i], qc);
+  }
+}
+
+// Persistent streaming version of the same: one CTA per SM, W warps, each warp walks over its
+// tokens with its own row buffer(s) in shared memory, filled by a bulk copy; while one warp waits
+// for its next row the others compute, so the HBM stream and the arithmetic overlap.  The row is read from
+// shared memory twice (sum of squares, then quantise); nothing is held in registers.
+// A wait on a row that does not arrive within about two seconds makes the warp stop (its
+// remaining tokens stay unwritten); nothing can be reported from here, the entry point has no
+// status word.
+__global__ void __launch_bounds__(1024) act_quant_stream_kernel(const ActQuantParams P, int W, int NB, uint32_t row_bytes) {
+  extern __shared__ __align__(128) uint8_t smem_aq[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  uint8_t* buf0 = smem_aq + (size_t)(warp * NB) * row_bytes;
+  const uint32_t bars = smem_u32(smem_aq + (size_t)(W * NB) * row_bytes) + (uint32_t)warp * 16u;
+  if (lane == 0) { mbar_init(bars, 1); mbar_init(bars + 8, 1); }
+  fence_mbar_init();
+  __syncthreads();
+  const int chunks = P.K >> 3;
+  const long long stride = (long long)gridDim.x * W;
+  const long long first = (long long)warp * gridDim.x + blockIdx.x;
+  const uint8_t* X = reinterpret_cast<const uint8_t*>(P.X);
+  const size_t ld_bytes = (size_t)P.ldx * 2;
+  if (lane == 0) {
+    for (int b = 0; b < NB; ++b) {
+      const long long t = first + b * stride;
+      if (t < P.M) {
+        mbar_arrive_expect_tx(bars + 8 * b, row_bytes);
+        bulk_load_1d(smem_u32(buf0 + (size_t)b * row_bytes), X + (size_t)t * ld_bytes, row_bytes, bars + 8 * b);
+      }
+    }
+  }
+  int it = 0;
+  for (long long t = first; t < P.M; t += stride, ++it) {
+    const int b = NB == 2 ? (it & 1) : 0; const uint32_t ph = (NB == 2 ? (it >> 1) : it) & 1;
+    {
+      const uint64_t t0 = globaltimer_ns();
+      bool ok = true;
+      while (!mbar_try_wait(bars + 8 * b, ph)) {
+        if (globaltimer_ns() - t0 > kWaitLimitNs) { ok = false; break; }
+      }
+      if (!__all_sync(0xffffffffu, ok)) return;
+    }
+    const uint4* row = reinterpret_cast<const uint4*>(buf0 + (size_t)b * row_bytes);
+    float r = 1.0f;
+    if (P.flags & FPT_RMSNORM) {
+      double acc0 = 0.0, acc1 = 0.0;
+      int c = lane;
+      for (; c + 32 < chunks; c += 64) { acc0 = sumsq(row[c], acc0); acc1 = sumsq(row[c + 32], acc1); }
+      if (c < chunks) acc0 = sumsq(row[c], acc0);
+      double acc = acc0 + acc1;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+      if (!((float)acc <= 3.4028234e38f)) {        // Inf / NaN in the row (or a genuine overflow): by the definition
+        acc = 0.0;
+        for (int c2 = lane; c2 < chunks; c2 += 32) acc = sumsq_exact(row[c2], acc);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+      }
+      const float ss = (float)acc;                 // one rounding to float32
+      const float ms = __fdiv_rn(ss, (float)P.K);
+      const float rho = __fsqrt_rn(__fadd_rn(ms, P.eps));
+      r = __fdiv_rn(1.0f, rho);
+    }
+    const float s = P.s_in ? __ldg(P.s_in + t) : 1.0f;
+    const float rs = P.s_in ? __fmul_rn(r, s) : r;
+    const float p = (P.flags & FPT_SCALE_INPUT) ? rs : r;
+    if (lane == 0) {
+      if (P.s_out) P.s_out[t] = rs;
+      if (P.post_inv) P.post_inv[t] = __fdiv_rn(1.0f, p);
+      if (P.r_out) P.r_out[t] = r;
+    }
+    uint32_t* out = P.Xq + (size_t)t * (size_t)chunks;
+    const QuantConsts qc = quant_consts(p, P);
+#pragma unroll 4
+    for (int c = lane; c < chunks; c += 32) out[c] = quant_word(row[c], qc);
+    __syncwarp();                                  // every lane is done with the buffer
+    const long long tn = t + NB * stride;
+    if (lane == 0 && tn < P.M) {
+      fence_proxy_async_smem();                    // our reads of the buffer come before the copy's writes
+      mbar_arrive_expect_tx(bars + 8 * b, row_bytes);
+      bulk_load_1d(smem_u32(buf0 + (size_t)b * row_bytes), X + (size_t)tn * ld_bytes, row_bytes, bars + 8 * b);
+    }
+  }
+}
+
+static cudaError_t launch_stream(const ActQuantParams& P, cudaStream_t st) {
+  static int sms = 0;
+  if (!sms) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (sms <= 0) sms = 1;
+    cudaError_t e = cudaFuncSetAttribute(act_quant_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+    if (e != cudaSuccess) { sms = 0; return e; }
+  }
+  // as many warps as row buffers fit (each warp needs at least one); two buffers per warp when
+  // 32 warps leave room for them
+  const uint32_t row_bytes = (uint32_t)P.K * 2;
+  const int fit = (int)((200u * 1024u) / row_bytes);
+  const int NB = fit >= 64 ? 2 : 1;
+  int wmax = fit / NB;
+  if (wmax > 32) wmax = 32;
+  const int grid = P.M < sms ? P.M : sms;
+  // warps per CTA: of the counts that fit, the one that leaves the fewest idle slots in the last
+  // round of tokens (a CTA gets about M / grid tokens, its warps take them in turns)
+  const int per_cta = (P.M + grid - 1) / grid;
+  int W = wmax; double best = 0.0;
+  for (int w = wmax; w >= 4 && 10 * w >= 7 * wmax; --w) {       // fewer warps also means less latency hiding
+    const int rounds = (per_cta + w - 1) / w;
+    const double eff = (double)per_cta / ((double)w * rounds);
+    if (eff > best + 0.1) { best = eff; W = w; }
+  }
+  const size_t smem = (size_t)W * NB * row_bytes + (size_t)W * 16;
+  act_quant_stream_kernel<<<grid, W * 32, smem, st>>>(P, W, NB, row_bytes);
+  return cudaGetLastError();
+}
+
+template <int V, int W>
+static cudaError_t launch_warp(const ActQuantParams& P, cudaStream_t st) {
+  act_quant_warp_kernel<V, W><<<(P.M + W - 1) / W, W * 32, 0, st>>>(P);
+  return cudaGetLastError();
 }
 
 template <int T, int V>
@@ -175,11 +434,18 @@ cudaError_t act_quant_launch(cudaStream_t st, const void* X, int M, int K, int l
   P.eps = eps;
   P.inv_delta = 1.0f / qp->scale;
   const int z = qp->symmetric ? 0 : qp->zero_point;
-  const int qmin = qp->symmetric ? -8 : 0, qmax = qp->symmetric ? 7 : 15;
-  P.lo = (float)(qmin - z);
-  P.hi = (float)(qmax - z);
-  P.magic = 12582912.0f + (float)z;
+  const int qmax = qp->symmetric ? 7 : 15;
+  P.qmax_minus_z = qmax - z;
+  P.flip = qp->symmetric ? 0x77777777u : 0xFFFFFFFFu;
   const int chunks = K / 8;
+  if (!(flags & FPT_SILU_MUL) && chunks >= 128 && chunks <= 2048 && M >= 512) return launch_stream(P, st);
+  if (!(flags & FPT_SILU_MUL)) {
+    if (chunks <= 64)        return launch_warp<2, 4>(P, st);
+    else if (chunks <= 128)  return launch_warp<4, 4>(P, st);
+    else if (chunks <= 256)  return launch_warp<8, 4>(P, st);
+    else if (chunks <= 512)  return launch_warp<16, 4>(P, st);
+    else if (chunks <= 1024) return launch_warp<32, 4>(P, st);
+  }
   if (chunks <= 128)        return launch<128, 1>(P, st);
   else if (chunks <= 256)   return launch<128, 2>(P, st);
   else if (chunks <= 512)   return launch<256, 2>(P, st);

@@ -34,6 +34,28 @@ def test_act_quant_codes_bit_exact(M, K, mode):
     assert len(np.unique(codes)) >= 8 or K < 64        # the grid is actually exercised
 
 
+@pytest.mark.parametrize("M,K,ld", [(600, 1024, 1024), (1500, 4096, 4096), (777, 8192, 8200), (513, 16384, 16384)])
+@pytest.mark.parametrize("mode", ["norm", "scale", "asym"])
+def test_act_quant_many_tokens_streaming_kernel(M, K, ld, mode):
+    """Enough tokens for the persistent double-buffered kernel: every warp walks over several rows,
+    some rows carry Inf / NaN / zeros, rows may be strided."""
+    x = torch.zeros((M, ld), dtype=torch.bfloat16)
+    x[:, :K] = _acts(M, K, 8)
+    x[:, K:] = -777.0
+    x[3, :K] = 0.0
+    x[M // 2, 11] = float("nan")
+    x[M - 1, K - 1] = float("inf")
+    s_in = synth.per_token_scale(M, 8, "s_in")
+    flags = B.SCALE_INPUT if mode == "scale" else B.RMSNORM
+    qp = B.QParams(4, mode != "asym", 0.37 if flags & B.RMSNORM else 1.9, 9)
+    xq, s_out = B.fpt_act_quant(dev(x), qp, flags, 1e-5, s_in=dev(s_in), K=K)
+    with np.errstate(all="ignore"):
+        codes, so, _, _ = OQ.act_quant(synth.f32(x)[:, :K], oqp(qp), bool(flags & B.RMSNORM),
+                                       bool(flags & B.SCALE_INPUT), 1e-5, s_in.numpy())
+    assert np.array_equal(host(xq), OQ.pack_int4(codes))
+    assert np.array_equal(host(s_out), so, equal_nan=True)
+
+
 def test_act_quant_strided_rows_and_edge_values():
     M, K, ld = 6, 256, 384
     x = torch.zeros((M, ld), dtype=torch.bfloat16)
@@ -43,6 +65,8 @@ def test_act_quant_strided_rows_and_edge_values():
     x[2, 5] = float("nan")
     x[3, 7] = float("inf")
     x[4, :K] = 3.0e38                                # squares overflow float32
+    x[5, 9] = 3.0e38                                 # finite, but far beyond the exact range of the rounding trick
+    x[5, 10] = -3.0e38
     qp = B.QParams(4, True, 0.41, 0)
     xq, s_out = B.fpt_act_quant(dev(x), qp, B.RMSNORM, 1e-6, K=K)
     with np.errstate(all="ignore"):
