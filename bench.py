@@ -31,6 +31,9 @@ M_TOK, HID, N_QKV, N_O = 2048, 4096, 6144, 4096
 D_FF = 14336
 EPS = 1e-5
 NSETS = 4
+# dram__bytes_read.sum + dram__bytes_write.sum of one fused-QKV matmul launch, from the ncu capture
+# summarised in profiles/ (None while the kernel has changed since its last capture)
+GEMM_QKV_DRAM_BYTES = None
 METRIC = "W4A4 linear TOPS (prefill, Llama-3-8B-shaped attention projections, 2048 tokens)"
 
 
@@ -217,18 +220,37 @@ def run_gpu(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for i in range(max(args.warmup, 3)):
-        step(sets[i % NSETS])
+    def capture(fn):
+        """One CUDA graph per operand set: the launches of `fn(S)` without the host's per-call cost."""
+        graphs = []
+        for S in sets:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                fn(S)
+            graphs.append(g)
+        return graphs
+
+    def timed(graphs, n):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(n):
+            graphs[i % NSETS].replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+
+    warm = max(args.warmup, 3)
+    for i in range(warm):
+        step(sets[i % NSETS])                        # eager: also sets the kernels' attributes before capture
+    torch.cuda.synchronize()
+    step_graphs = capture(step)
+    for i in range(NSETS):
+        step_graphs[i].replay()
     barrier()
     sampler = ClockSampler(local)
     sampler.start()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for i in range(args.steps):
-        step(sets[i % NSETS])
-    e1.record()
+    ms = timed(step_graphs, args.steps)
     barrier()
-    ms = e0.elapsed_time(e1)
     clocks = sampler.result()
     for S in sets:
         assert B.fpt_check_status(S["ws1"]) == B.OK and B.fpt_check_status(S["ws2"]) == B.OK
@@ -239,7 +261,7 @@ def run_gpu(args):
     ms_per_step = ms / args.steps
     tops = world * step_ops("attn") / (ms_per_step * 1e-3) / 1e12
 
-    # ---- end to end: host buffers in, results back, every step ------------------------------
+    # ---- end to end: host buffers in, results back, every step (eager calls through the binding) ----
     h_y1 = torch.empty((M_TOK, N_QKV), dtype=torch.bfloat16).pin_memory()
     h_y2 = torch.empty((M_TOK, N_O), dtype=torch.bfloat16).pin_memory()
     e2e_steps = max(3, min(args.steps, 50))
@@ -254,6 +276,7 @@ def run_gpu(args):
     for i in range(3):
         e2e_step(sets[i % NSETS])
     barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for i in range(e2e_steps):
         e2e_step(sets[i % NSETS])
@@ -268,26 +291,25 @@ def run_gpu(args):
     h2d = 2 * M_TOK * HID * 2
     d2h = M_TOK * (N_QKV + N_O) * 2
 
-    # ---- per-kernel pass: the same step as separate C-ABI calls with events around each -------
-    ksteps = max(8, min(args.steps, 200))
-    names = ["act_quant_x", "gemm_qkv", "act_quant_ao", "gemm_o"]
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(ksteps)]
+    # ---- per-kernel pass: each of the step's four kernels alone, replayed over the rotating sets ----
+    ksteps = max(8, min(args.steps, 400))
     xq = [torch.empty((M_TOK, HID // 2), dtype=torch.uint8, device=dev) for _ in range(2)]
     gws = B.new_workspace(B.OP_GEMM, M_TOK, N_QKV, HID, dev)
-    for i in range(ksteps + 3):
-        S = sets[i % NSETS]
-        ev = evs[max(i - 3, 0)]
-        ev[0].record()
-        B.fpt_act_quant(S["x"], qp_x, B.RMSNORM, EPS, want_s_out=False, out=xq[0])
-        ev[1].record()
-        B.fpt_w4a4_gemm(xq[0], S["wq1"], S["sw1"], qp_x.scale, ws=gws, Y=S["y1"])
-        ev[2].record()
-        B.fpt_act_quant(S["ao"], qp_o, B.SCALE_INPUT, EPS, s_in=S["s_in"], want_s_out=False, out=xq[1])
-        ev[3].record()
-        B.fpt_w4a4_gemm(xq[1], S["wq2"], S["sw2"], qp_o.scale, ws=gws, Y=S["y2"])
-        ev[4].record()
+    B.fpt_act_quant(sets[0]["x"], qp_x, B.RMSNORM, EPS, want_s_out=False, out=xq[0])
+    B.fpt_act_quant(sets[0]["ao"], qp_o, B.SCALE_INPUT, EPS, s_in=sets[0]["s_in"], want_s_out=False, out=xq[1])
     torch.cuda.synchronize()
-    kern_us = {n: float(np.mean([ev[j].elapsed_time(ev[j + 1]) for ev in evs])) * 1e3 for j, n in enumerate(names)}
+    kernels = {
+        "act_quant_x": lambda S: B.fpt_act_quant(S["x"], qp_x, B.RMSNORM, EPS, want_s_out=False, out=xq[0]),
+        "gemm_qkv": lambda S: B.fpt_w4a4_gemm(xq[0], S["wq1"], S["sw1"], qp_x.scale, ws=gws, Y=S["y1"]),
+        "act_quant_ao": lambda S: B.fpt_act_quant(S["ao"], qp_o, B.SCALE_INPUT, EPS, s_in=S["s_in"], want_s_out=False,
+                                                  out=xq[1]),
+        "gemm_o": lambda S: B.fpt_w4a4_gemm(xq[1], S["wq2"], S["sw2"], qp_o.scale, ws=gws, Y=S["y2"]),
+    }
+    kern_us = {}
+    for name, fn in kernels.items():
+        gs = capture(fn)
+        timed(gs, NSETS)
+        kern_us[name] = timed(gs, ksteps) * 1e3 / ksteps
     peaks = load_peaks()
     long_run = ms > 2000.0
     bf16_peak = peaks["bf16_sustained"] if long_run else peaks["bf16_burst"]
@@ -295,11 +317,11 @@ def run_gpu(args):
     gemm_ops = 2.0 * M_TOK * HID * N_QKV
     achieved = gemm_ops / (kern_us["gemm_qkv"] * 1e-6) / 1e12
     aq_bytes = M_TOK * HID * 2.5 + M_TOK * 4
-    roofline = {"kernel": "gemm_w4a4_kernel<256> (fused QKV, 2048x6144x4096)", "bound": "tensor",
-                "achieved": achieved, "peak": int8_peak, "unit": "TOP/s", "frac": achieved / int8_peak,
-                "traffic": None,
+    roofline = {"kernel": "gemm_w4a4_pair_kernel (fused QKV, 2048x6144x4096, CTA pairs, 256x256 tiles)",
+                "bound": "tensor", "achieved": achieved, "peak": int8_peak, "unit": "TOP/s",
+                "frac": achieved / int8_peak, "traffic": GEMM_QKV_DRAM_BYTES,
                 "peak_note": f"2 x {peaks['source']} bf16 {'sustained' if long_run else 'burst'} peak "
-                             f"({bf16_peak} TFLOP/s); nominal dense int8 is 4500",
+                             f"({bf16_peak} TFLOP/s), the nominal int8 : bf16 ratio; nominal dense int8 is 4500",
                 "frac_of_nominal_4500": achieved / 4500.0,
                 "act_quant": {"bound": "hbm", "achieved": aq_bytes / (kern_us["act_quant_x"] * 1e-6) / 1e9,
                               "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -319,8 +341,8 @@ def run_gpu(args):
                                  f"(> 126 MB L2 in total)"},
                 "e2e": {"value": e2e_tops, "unit": "TOPS", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                         "steps": e2e_steps},
-                "gpu_launches": 4 * args.steps, "clocks": clocks, "roofline": roofline,
-                "kernel_us": kern_us,
+                "gpu_launches": 4 * args.steps, "launch_mode": "one CUDA graph per step (4 kernels), replayed",
+                "clocks": clocks, "roofline": roofline, "kernel_us": kern_us,
                 "cpu_baseline": {"value": cpu_tops, "unit": "TOPS", "cores": blas_threads(), "kind": "oracle",
                                  "sample": f"{rows} of {M_TOK} token rows x all {N_QKV + N_O} output columns, "
                                            f"8 repetitions, {cpu_dt:.2f} s each"}}
