@@ -298,6 +298,13 @@ __device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const uint32_t* v)
       : "memory");
 }
 
+// Register re-allocation between warpgroups (4 consecutive warps, all must execute it): a group
+// that needs few registers gives some back, another takes them.  N is a multiple of 8.  A CTA can
+// only redistribute the registers it was launched with: an increase that the decreases of the
+// other groups do not cover never returns.
+template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+
 __device__ __forceinline__ void named_bar_sync(uint32_t id, uint32_t nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }

@@ -128,7 +128,14 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
   tc_fence_after();
   const uint32_t tmem_base = misc[0];
 
-  if (warp == 0) {
+  // Registers: the epilogue wants the 128 accumulators of its row in registers at once, the other
+  // roles need few; the warpgroups trade.  A CTA can only redistribute what it was launched with
+  // (640 x 96 registers): 128 x (48 + 56 + 56) + 256 x 152 = 59392 <= 61440, so the request of the
+  // epilogue groups is always met once the three other groups have given theirs back.  Each role
+  // branch starts with its own re-allocation (the compiler budgets registers per branch).
+  if (warp < kConvAWarp0) {
+    reg_dec<48>();
+    if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       int s = 0; uint32_t ph = 0;
@@ -155,7 +162,7 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             while (!mbar_try_wait(pk_full(q), (armed_par >> q) & 1u) && globaltimer_ns() - t0 < 2000000ull) {}
       }
     }
-  } else if (warp == 1) {
+    } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA only)
     if (rank == 0 && lane == 0) {
       const uint32_t idesc = umma_idesc_i8(TM, TN, !P.a_unsigned, true);
@@ -179,8 +186,10 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         umma_commit_pair(acc_full, 3);
       }
     }
-  } else if (warp >= kConvAWarp0 && warp < kConvBWarp0) {
+    }
+  } else if (warp < kConvBWarp0) {
     // ------------------------------------------------------------------ activation converters -> tensor memory
+    reg_dec<56>();
     const int quad = warp - kConvAWarp0;                 // == warp % 4: the TMEM lanes this warp may touch
     const int r = quad * 32 + lane;                      // row of the CTA's 128
     const uint32_t swz = (uint32_t)((r >> 1) & 3);       // SWIZZLE_64B: 16-byte chunk index ^= (row / 2) % 4
@@ -210,8 +219,9 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         if (++s == NS) { s = 0; ph ^= 1u; }
       }
     }
-  } else if (warp >= kConvBWarp0 && warp < kEpiWarp0) {
+  } else if (warp < kEpiWarp0) {
     // ------------------------------------------------------------------ weight converters -> shared int8 tile
+    reg_dec<56>();
     const int ctid = threadIdx.x - kConvBWarp0 * 32;     // 0..127
     const uint32_t op_full_leader = map_to_cta(op_full(0), 0);
     int ps = 0, s = 0; uint32_t pph = 0, ph = 0;
@@ -244,8 +254,9 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         if (++s == NS) { s = 0; ph ^= 1u; }
       }
     }
-  } else if (warp >= kEpiWarp0) {
+  } else {
     // ------------------------------------------------------------------ epilogue
+    reg_inc<152>();
     const int quad = warp & 3;                           // TMEM lane quadrant this warp may read
     const int half = (warp - kEpiWarp0) >> 2;            // which 128 of the 256 columns
     const int etid = (warp - kEpiWarp0) * 32 + lane;     // 0..255: the tile column whose scale this thread fetches
@@ -282,18 +293,25 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
       const size_t rowoff = (size_t)row * (size_t)P.N;
       const float* sws = sw_s + b * TN + half * 128;
       const int* zws = zw_s + b * TN + half * 128;
-#pragma unroll 1
+      // all 128 accumulators of this thread's row -> registers, then the accumulator is free again
+      uint32_t v[128];
+      tmem_ld_32x32(taddr, *reinterpret_cast<uint32_t(*)[32]>(v));
+      tmem_ld_32x32(taddr + 32, *reinterpret_cast<uint32_t(*)[32]>(v + 32));
+      tmem_ld_32x32(taddr + 64, *reinterpret_cast<uint32_t(*)[32]>(v + 64));
+      tmem_ld_32x32(taddr + 96, *reinterpret_cast<uint32_t(*)[32]>(v + 96));
+      tmem_wait_ld();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
+#pragma unroll
       for (int ch = 0; ch < 4; ++ch) {
-        uint32_t v[32];
-        tmem_ld_32x32(taddr + ch * 32, v);
-        tmem_wait_ld();
         uint8_t* slab = smem + L::kStgOff + (half * 2 + (ch >> 1)) * L::kStgSlab + r * 128;
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
           const int col = nt + half * 128 + ch * 32 + g * 8;
           int a[8];
 #pragma unroll
-          for (int j = 0; j < 8; ++j) a[j] = (((int)v[g * 8 + j]) >> 8) - zws[ch * 32 + g * 8 + j];
+          for (int j = 0; j < 8; ++j) a[j] = (((int)v[ch * 32 + g * 8 + j]) >> 8) - zws[ch * 32 + g * 8 + j];
           if (P.acc_out && row_ok && col < P.N) {
             int4* o = reinterpret_cast<int4*>(P.acc_out + rowoff + col);
             o[0] = make_int4(a[0], a[1], a[2], a[3]);
@@ -326,10 +344,6 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
           }
         }
       }
-      // the accumulator has been read: the next tile's matmul may overwrite it
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
       if (P.Y) {
         fence_proxy_async_smem();                        // staged tile -> visible to the TMA engine
         __syncwarp();
