@@ -44,6 +44,36 @@ def step_ops(workload):
 
 
 # ------------------------------------------------------------------------------------------
+# multi-rank bookkeeping (the path has no exchange step: every rank runs its own token shard)
+# ------------------------------------------------------------------------------------------
+def rank_info():
+    """(rank, world, local rank) from the launcher's environment."""
+    return (int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1")),
+            int(os.environ.get("LOCAL_RANK", "0")))
+
+
+def shard_tag(i, rank):
+    """Name suffix of operand set i of a rank: every rank draws its own tokens and weights copies."""
+    return f"{i + NSETS * rank}"
+
+
+def max_over_ranks(ms, world, device):
+    """The slowest rank's time: the job is done when the last rank is."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(ops_per_step, world, ms_per_step):
+    """Whole-job TOP/s: all ranks' work over the slowest rank's time."""
+    return world * ops_per_step / (ms_per_step * 1e-3) / 1e12
+
+
+# ------------------------------------------------------------------------------------------
 # clocks
 # ------------------------------------------------------------------------------------------
 class ClockSampler(threading.Thread):
@@ -131,7 +161,7 @@ def time_oracle(rows, reps):
 
 
 def run_reference(args):
-    rank = int(os.environ.get("RANK", "0"))
+    rank, _, _ = rank_info()
     if rank != 0:
         return
     # size the per-step sample so that warmup + steps end within about two minutes
@@ -179,9 +209,7 @@ def run_gpu(args):
     import torch.distributed as dist
     from paper_2506_04985_b200 import binding as B, synth, build
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = rank_info()
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl")
@@ -192,7 +220,7 @@ def run_gpu(args):
     # ---- seeded inputs: NSETS rotating sets so that every step reads HBM, not L2 ------------
     sets = []
     for i in range(NSETS):
-        tag = f"{i + NSETS * rank}"
+        tag = shard_tag(i, rank)
         x = synth.activations(M_TOK, HID, 0, "bench/x" + tag, law="student_t3", outlier_frac=0.005, outlier_gain=50.0)
         ao = synth.activations(M_TOK, HID, 0, "bench/ao" + tag, law="student_t3", outlier_frac=0.005, outlier_gain=50.0)
         s_in = synth.per_token_scale(M_TOK, 0, "bench/s" + tag)
@@ -254,12 +282,9 @@ def run_gpu(args):
     clocks = sampler.result()
     for S in sets:
         assert B.fpt_check_status(S["ws1"]) == B.OK and B.fpt_check_status(S["ws2"]) == B.OK
-    if world > 1:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, world, dev)
     ms_per_step = ms / args.steps
-    tops = world * step_ops("attn") / (ms_per_step * 1e-3) / 1e12
+    tops = job_throughput(step_ops("attn"), world, ms_per_step)
 
     # ---- end to end: host buffers in, results back, every step (eager calls through the binding) ----
     h_y1 = torch.empty((M_TOK, N_QKV), dtype=torch.bfloat16).pin_memory()
@@ -283,11 +308,8 @@ def run_gpu(args):
     e1.record()
     barrier()
     ms_e2e = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms_e2e], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
-    e2e_tops = world * step_ops("attn") / (ms_e2e / e2e_steps * 1e-3) / 1e12
+    ms_e2e = max_over_ranks(ms_e2e, world, dev)
+    e2e_tops = job_throughput(step_ops("attn"), world, ms_e2e / e2e_steps)
     h2d = 2 * M_TOK * HID * 2
     d2h = M_TOK * (N_QKV + N_O) * 2
 
