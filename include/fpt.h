@@ -65,7 +65,7 @@ extern "C" {
 #define FPT_RMSNORM         1     /* r_t = 1/sqrt(mean_k x^2 + eps); the grid sees x * r_t        */
 #define FPT_SCALE_INPUT     2     /* the grid sees x * s_in[t] (times r_t when FPT_RMSNORM too)   */
 #define FPT_SILU_MUL        4     /* x := bf16(silu(X) * X2) before anything else (no RMSNORM)    */
-#define FPT_GU_INTERLEAVED  8     /* with FPT_SILU_MUL: X holds gate||up in 128-column groups     */
+#define FPT_GU_INTERLEAVED  8     /* with FPT_SILU_MUL: X holds gate||up in 64-column groups      */
 
 /* where the per-token scale ends up after the matmul (Sec. 3.1.3: the scale commutes
  * with a bias-free linear, so the caller chooses) */
@@ -110,11 +110,12 @@ int fpt_quantize_weights(void* stream, const void* W, int w_dtype, int N, int K,
 
 /*
  * Copies separately quantised gate and up matrices into the row-interleaved layout that
- * fpt_decoder_mlp expects: for every group r of 128 output features, rows
- * [256 r, 256 r + 128) of Wgu_q are gate rows [128 r, 128 r + 128) and rows
- * [256 r + 128, 256 r + 256) are the matching up rows; sw_gu follows the same order.
- * d_ff must be a multiple of 128.  (No counterpart in the paper: it is a storage choice
- * that lets one matmul tile hold a gate column and its up column.)
+ * fpt_decoder_mlp expects: for every group r of 64 output features, rows
+ * [128 r, 128 r + 64) of Wgu_q are gate rows [64 r, 64 r + 64) and rows
+ * [128 r + 64, 128 r + 128) are the matching up rows; sw_gu follows the same order.
+ * d_ff must be a multiple of 64.  (No counterpart in the paper: it is a storage choice
+ * that puts a gate column and its up column into the registers of one epilogue thread, so
+ * that the SwiGLU product and the next quantiser run inside the matmul.)
  */
 int fpt_interleave_gate_up(void* stream, const uint8_t* Wg_q, const uint8_t* Wu_q,
                            const void* sw_g, const void* sw_u, int scale_dtype,
@@ -134,7 +135,7 @@ int fpt_interleave_gate_up(void* stream, const uint8_t* Wg_q, const uint8_t* Wu_
  *   X      [M, ldx] bf16, ldx >= K elements, ldx % 8 == 0
  *   X2     second operand of FPT_SILU_MUL, same layout as X; with FPT_GU_INTERLEAVED X2 is
  *          ignored, X is [M, 2K] (ldx >= 2K) and logical column k lives at
- *          gate: (k/128)*256 + k%128, up: gate + 128
+ *          gate: (k/64)*128 + k%64, up: gate + 64
  *   s_in   [M] f32 or NULL;  s_out [M] f32 or NULL
  *   Xq     [M, K/2] packed codes out
  * silu(g) = g / (1 + 2^(-g*log2 e)) with a fixed float32 polynomial for 2^f (degree 6

@@ -4,6 +4,7 @@
 // with 128-bit loads, kept in registers across the reduction, and written as packed
 // nibbles.
 #include "fpt_internal.cuh"
+#include "quant_math.cuh"
 
 namespace fpt {
 
@@ -22,98 +23,6 @@ struct ActQuantParams {
   int   qmax_minus_z;  // upper end of the grid minus the zero point
   uint32_t flip;       // see quant_word
 };
-
-// 2^f on [-0.5, 0.5]: degree-6 Taylor coefficients (ln 2)^k / k!, rounded to float32.
-__device__ __forceinline__ float exp2_spec(float t) {
-  t = fminf(fmaxf(t, -126.0f), 126.0f);
-  const float n = rintf(t);
-  const float f = __fsub_rn(t, n);
-  float a = 0x1.430912p-13f;                               // (ln2)^6 / 720
-  a = __fadd_rn(__fmul_rn(a, f), 0x1.5d87fep-10f);         // (ln2)^5 / 120
-  a = __fadd_rn(__fmul_rn(a, f), 0x1.3b2ab6p-7f);          // (ln2)^4 / 24
-  a = __fadd_rn(__fmul_rn(a, f), 0x1.c6b08ep-5f);          // (ln2)^3 / 6
-  a = __fadd_rn(__fmul_rn(a, f), 0x1.ebfbep-3f);           // (ln2)^2 / 2
-  a = __fadd_rn(__fmul_rn(a, f), 0x1.62e43p-1f);           // ln2
-  a = __fadd_rn(__fmul_rn(a, f), 1.0f);
-  const float two_n = __int_as_float(((int)n + 127) << 23);
-  return __fmul_rn(a, two_n);
-}
-
-__device__ __forceinline__ float silu_spec(float g) {
-  const float e = exp2_spec(__fmul_rn(-g, 0x1.715476p+0f));   // log2(e)
-  return __fdiv_rn(g, __fadd_rn(1.0f, e));
-}
-
-// bf16(silu(g) * u) for a packed pair of bf16 values.
-__device__ __forceinline__ uint32_t silu_mul_pair(uint32_t g, uint32_t u) {
-  const float lo = __fmul_rn(silu_spec(bf16lo_to_f32(g)), bf16lo_to_f32(u));
-  const float hi = __fmul_rn(silu_spec(bf16hi_to_f32(g)), bf16hi_to_f32(u));
-  return f32_to_bf16_bits(lo) | (f32_to_bf16_bits(hi) << 16);
-}
-
-// Two float32 lanes in one 64-bit register: sm_100 multiplies both with one instruction, each
-// lane rounded to nearest even on its own (the same result as two scalar multiplies).
-__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
-  uint64_t r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-  return r;
-}
-__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ uint64_t mul_f32x2(uint64_t a, uint64_t b) {
-  uint64_t r;
-  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-  return r;
-}
-__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
-  uint64_t r;
-  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-  return r;
-}
-
-// Quantiser arithmetic of one 16-byte chunk (8 values), in the order the header states:
-//   u = (x * p) * (1/D)          two separately rounded float32 multiplies
-//   q = clamp(rne(u) + z)        a NaN maps to the lowest code
-// evaluated on the NEGATED value v = (x * -p) * (1/D) = -u (negation is exact and rounding to
-// nearest even is symmetric): adding 1.5 * 2^23 leaves -rne(u) in the low mantissa bits, and the
-// float's bit pattern is monotone in v, also beyond the exact range and for +Inf and NaN, which
-// are the largest patterns.  One integer add-min-relu then yields qmax - q in [0, 15] with the
-// NaN at qmax - qmin = 15, i.e. the lowest code; the nibbles are flipped back by one XOR per
-// word (15 - c = c ^ 15; on the symmetric grid the two's complement nibble of 7 - c is c ^ 7).
-struct QuantConsts {
-  uint64_t np2, d2, m2;   // (-p, -p), (1/D, 1/D), (magic, magic)
-  int bias;               // -(bits of magic) + (qmax - z)
-  uint32_t flip;          // 0x77777777 symmetric, 0xFFFFFFFF asymmetric
-};
-
-__device__ __forceinline__ QuantConsts quant_consts(float p, const ActQuantParams& P) {
-  QuantConsts c;
-  c.np2 = pack_f32x2(-p, -p);
-  c.d2 = pack_f32x2(P.inv_delta, P.inv_delta);
-  c.m2 = pack_f32x2(12582912.0f, 12582912.0f);
-  c.bias = -0x4B400000 + P.qmax_minus_z;
-  c.flip = P.flip;
-  return c;
-}
-
-// Two values of one 32-bit word -> (15 - code) each, the second in front: returns c0 + 16 * c1 + 256 * prev.
-__device__ __forceinline__ uint32_t quant_pair(uint32_t w, const QuantConsts& c, uint32_t prev) {
-  float v0, v1;
-  unpack_f32x2(add_f32x2(mul_f32x2(mul_f32x2(pack_f32x2(bf16lo_to_f32(w), bf16hi_to_f32(w)), c.np2), c.d2), c.m2), v0, v1);
-  // (a negative sum -- u beyond 1.2e7 -- has a negative pattern; max(., 0) keeps the add below from wrapping)
-  const uint32_t c0 = (uint32_t)__viaddmin_s32_relu(max(__float_as_int(v0), 0), c.bias, 15);
-  const uint32_t c1 = (uint32_t)__viaddmin_s32_relu(max(__float_as_int(v1), 0), c.bias, 15);
-  return (prev * 16u + c1) * 16u + c0;
-}
-
-__device__ __forceinline__ uint32_t quant_word(const uint4& v, const QuantConsts& c) {
-  uint32_t w = quant_pair(v.w, c, 0u);
-  w = quant_pair(v.z, c, w);
-  w = quant_pair(v.y, c, w);
-  w = quant_pair(v.x, c, w);
-  return w ^ c.flip;
-}
 
 // acc + the 8 squares of a chunk in float64.  The bf16 magnitude bits, moved to the top of a
 // float64's high word, are the value times 2^-896 for every finite input (normal, subnormal or
@@ -165,10 +74,10 @@ __global__ void __launch_bounds__(T) act_quant_kernel(const ActQuantParams P) {
       if (!silu) {
         v[i] = __ldg(P.X + row + c);
       } else {
-        // gate column of logical chunk c: groups of 16 chunks (128 columns), gate then up
-        const int gc = inter ? ((c >> 4) << 5) + (c & 15) : c;
+        // gate column of logical chunk c: groups of 8 chunks (64 columns), gate then up
+        const int gc = inter ? ((c >> 3) << 4) + (c & 7) : c;
         const uint4 g = __ldg(P.X + row + gc);
-        const uint4 u = inter ? __ldg(P.X + row + gc + 16) : __ldg(P.X2 + row + c);
+        const uint4 u = inter ? __ldg(P.X + row + gc + 8) : __ldg(P.X2 + row + c);
         v[i].x = silu_mul_pair(g.x, u.x);
         v[i].y = silu_mul_pair(g.y, u.y);
         v[i].z = silu_mul_pair(g.z, u.z);
@@ -226,7 +135,7 @@ __global__ void __launch_bounds__(T) act_quant_kernel(const ActQuantParams P) {
     if (P.r_out) P.r_out[t] = r;
   }
   uint32_t* out = P.Xq + (size_t)t * (size_t)chunks;
-  const QuantConsts qc = quant_consts(p, P);
+  const QuantConsts qc = quant_consts(p, P.inv_delta, P.qmax_minus_z, P.flip);
 #pragma unroll
   for (int i = 0; i < V; ++i) {
     const int c = i * T + tid;
@@ -281,7 +190,7 @@ __global__ void __launch_bounds__(W * 32) act_quant_warp_kernel(const ActQuantPa
     if (P.r_out) P.r_out[t] = r;
   }
   uint32_t* out = P.Xq + (size_t)t * (size_t)chunks;
-  const QuantConsts qc = quant_consts(p, P);
+  const QuantConsts qc = quant_consts(p, P.inv_delta, P.qmax_minus_z, P.flip);
 #pragma unroll
   for (int i = 0; i < V; ++i) {
     const int c = i * 32 + lane;
@@ -359,7 +268,7 @@ __global__ void __launch_bounds__(1024) act_quant_stream_kernel(const ActQuantPa
       if (P.r_out) P.r_out[t] = r;
     }
     uint32_t* out = P.Xq + (size_t)t * (size_t)chunks;
-    const QuantConsts qc = quant_consts(p, P);
+    const QuantConsts qc = quant_consts(p, P.inv_delta, P.qmax_minus_z, P.flip);
 #pragma unroll 4
     for (int c = lane; c < chunks; c += 32) out[c] = quant_word(row[c], qc);
     __syncwarp();                                  // every lane is done with the buffer
@@ -471,7 +380,7 @@ extern "C" int fpt_act_quant(void* stream, const void* X, int M, int K, int ldx,
   if (inter && !silu) return FPT_ERR_BAD_ARG;
   if (silu && (flags & FPT_RMSNORM)) return FPT_ERR_UNSUPPORTED;
   if (silu && !inter && !X2) return FPT_ERR_BAD_ARG;
-  if (inter && K % 128 != 0) return FPT_ERR_UNSUPPORTED;
+  if (inter && K % 64 != 0) return FPT_ERR_UNSUPPORTED;
   if ((flags & FPT_SCALE_INPUT) && !s_in) return FPT_ERR_BAD_ARG;
   const int need_ld = inter ? 2 * K : K;
   if (ldx < need_ld || ldx % 8 != 0) return FPT_ERR_ALIGNMENT;

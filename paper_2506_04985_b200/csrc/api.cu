@@ -161,14 +161,30 @@ extern "C" int fpt_decoder_mlp(void* stream, const void* X, int M, int d, int d_
   // X~ = RMSNorm(X) on the grid qp_in; S_n = S_{n-1} * r
   if (act_quant_launch(st, X, M, d, d, qp_in, FPT_RMSNORM, eps, nullptr, s_prev, Xq, sn, nullptr, r_ws) != cudaSuccess)
     return FPT_ERR_CUDA;
-  // gate || up in one matmul over the interleaved weight
-  rc = fpt_w4a4_gemm(stream, Xq, Wgu_q, M, 2 * d_ff, d, sw_gu, scale_dtype, nullptr, qp_in->scale, 1, 0, nullptr,
-                     nullptr, nullptr, GU, nullptr, workspace, gemm_ws);
-  if (rc) return rc;
-  // m = bf16(silu(g) * u), quantised after the multiply by S_n
-  if (act_quant_launch(st, GU, M, d_ff, 2 * d_ff, qp_mid, FPT_SILU_MUL | FPT_GU_INTERLEAVED | FPT_SCALE_INPUT, 0.0f,
-                       nullptr, sn, Mq, nullptr, nullptr, nullptr) != cudaSuccess)
-    return FPT_ERR_CUDA;
+  if (M > 128 && (((uintptr_t)sw_gu | (uintptr_t)sw_d) & 15) == 0) {
+    // gate || up in one matmul whose epilogue forms m = bf16(silu(g) * u) and quantises m * S_n:
+    // the static grid and S_n are known before the matmul starts, so g and u never reach memory
+    GemmParams P{};
+    P.M = M; P.N = 2 * d_ff; P.K = d;
+    P.sw = sw_gu; P.scale_dtype = scale_dtype;
+    P.act_scale = qp_in->scale;
+    P.Mq = Mq; P.mid_scale = sn;
+    P.mid_inv_delta = 1.0f / qp_mid->scale;
+    P.mid_qmax_minus_z = 7; P.mid_flip = 0x77777777u;
+    P.status = reinterpret_cast<uint32_t*>(workspace);
+    P.scratch = ws + kStatusBytes;
+    rc = gemm_pair_launch(st, Xq, Wgu_q, P);
+    if (rc) return rc;
+  } else {
+    // gate || up in one matmul over the interleaved weight
+    rc = fpt_w4a4_gemm(stream, Xq, Wgu_q, M, 2 * d_ff, d, sw_gu, scale_dtype, nullptr, qp_in->scale, 1, 0, nullptr,
+                       nullptr, nullptr, GU, nullptr, workspace, gemm_ws);
+    if (rc) return rc;
+    // m = bf16(silu(g) * u), quantised after the multiply by S_n
+    if (act_quant_launch(st, GU, M, d_ff, 2 * d_ff, qp_mid, FPT_SILU_MUL | FPT_GU_INTERLEAVED | FPT_SCALE_INPUT, 0.0f,
+                         nullptr, sn, Mq, nullptr, nullptr, nullptr) != cudaSuccess)
+      return FPT_ERR_CUDA;
+  }
   // down projection; the normalised residual X * r joins before the final rounding
   return fpt_w4a4_gemm(stream, Mq, Wd_q, M, d, d_ff, sw_d, scale_dtype, nullptr, qp_mid->scale, 1, 0, nullptr,
                        add_residual ? X : nullptr, add_residual ? r_ws : nullptr, Y, nullptr, workspace, gemm_ws);

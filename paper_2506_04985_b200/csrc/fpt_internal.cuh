@@ -19,6 +19,14 @@ struct GemmParams {
   const float* res_scale;
   __nv_bfloat16* Y;
   int32_t* acc_out;
+  // SwiGLU + quantise fused into the epilogue (gate||up matmul of the MLP block, CTA-pair kernel
+  // only): with Mq set, the columns are 64 gate | 64 up | ... output features, no bf16 tile is
+  // written, and m = bf16(silu(g) * u) is quantised with the per-token multiplier mid_scale[t]
+  uint8_t* Mq;                 // [M, N/4] packed codes of the N/2 products, or nullptr
+  const float* mid_scale;      // [M] S_n
+  float mid_inv_delta;         // 1/D of the grid at the down-projection input
+  int mid_qmax_minus_z;
+  uint32_t mid_flip;
   uint32_t* status;            // control block of the workspace (status word, decode counters)
   void* scratch;               // gemm_scratch_bytes(M) bytes behind the control block (decode partial sums)
 };

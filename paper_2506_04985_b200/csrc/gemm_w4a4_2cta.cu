@@ -24,6 +24,7 @@
 #include <cuda.h>
 
 #include "fpt_internal.cuh"
+#include "quant_math.cuh"
 
 namespace fpt {
 namespace pair {
@@ -117,7 +118,7 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     fence_mbar_init();
     prefetch_tmap(&tmA);
     prefetch_tmap(&tmB);
-    if (P.Y) prefetch_tmap(&tmY);
+    if (P.Y || P.Mq) prefetch_tmap(&tmY);
   }
   if (warp == 1) {
     tmem_alloc_pair(sbase + L::kMiscOff, kTmemCols);
@@ -282,11 +283,12 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
       float c = P.act_scale, rs = 1.0f;
       if (row_ok && P.post) c = __fmul_rn(P.act_scale, __ldg(P.post + row));
       if (row_ok && P.res_scale) rs = __ldg(P.res_scale + row);
+      const float sn = (P.Mq && row_ok) ? __ldg(P.mid_scale + row) : 0.0f;
       __syncwarp();
       if (lane == 0) mbar_arrive(sc_full(b));
       if (!mbar_wait(sc_full(b), bph, abort_flag, P.status, 9)) break;
       // the staging half must have been read by the TMA store of the previous tile
-      if (P.Y && !mbar_wait(stg_empty(half), (it & 1) ^ 1u, abort_flag, P.status, 10)) break;
+      if ((P.Y || P.Mq) && !mbar_wait(stg_empty(half), (it & 1) ^ 1u, abort_flag, P.status, 10)) break;
       if (!mbar_wait(acc_full, it & 1, abort_flag, P.status, 4)) break;
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + half * 128;
@@ -303,6 +305,34 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
+      if (P.Mq) {
+        // v[0..63]: gate accumulators of 64 features, v[64..127]: their up accumulators.
+        // g, u = bf16 outputs of the two linears; m = bf16(silu(g) * u); code = grid(m * S_n).
+        const QuantConsts qc = quant_consts(sn, P.mid_inv_delta, P.mid_qmax_minus_z, P.mid_flip);
+        uint32_t codes[8];
+#pragma unroll
+        for (int j8 = 0; j8 < 8; ++j8) {
+          uint32_t mw[4];
+#pragma unroll
+          for (int jj = 0; jj < 4; ++jj) {
+            const int f = j8 * 8 + jj * 2;
+            uint32_t gw = 0, uw = 0;
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              const int ag = ((int)v[f + e]) >> 8, au = ((int)v[64 + f + e]) >> 8;
+              const float gf = magic_ok ? __fsub_rn(__int_as_float(0x4B400000 + ag), 12582912.0f) : (float)ag;
+              const float uf = magic_ok ? __fsub_rn(__int_as_float(0x4B400000 + au), 12582912.0f) : (float)au;
+              gw |= f32_to_bf16_bits(__fmul_rn(__fmul_rn(gf, sws[f + e]), c)) << (16 * e);
+              uw |= f32_to_bf16_bits(__fmul_rn(__fmul_rn(uf, sws[64 + f + e]), c)) << (16 * e);
+            }
+            mw[jj] = silu_mul_pair(gw, uw);
+          }
+          codes[j8] = quant_word(make_uint4(mw[0], mw[1], mw[2], mw[3]), qc);
+        }
+        uint4* stg = reinterpret_cast<uint4*>(smem + L::kStgOff + (half * 2) * L::kStgSlab + r * 32);
+        stg[0] = make_uint4(codes[0], codes[1], codes[2], codes[3]);
+        stg[1] = make_uint4(codes[4], codes[5], codes[6], codes[7]);
+      } else {
 #pragma unroll
       for (int ch = 0; ch < 4; ++ch) {
         uint8_t* slab = smem + L::kStgOff + (half * 2 + (ch >> 1)) * L::kStgSlab + r * 128;
@@ -344,15 +374,20 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
           }
         }
       }
-      if (P.Y) {
+      }
+      if (P.Y || P.Mq) {
         fence_proxy_async_smem();                        // staged tile -> visible to the TMA engine
         __syncwarp();
         if (lane == 0) mbar_arrive(stg_full(half));
         if (issuer) {
           if (!mbar_wait(stg_full(half), it & 1, abort_flag, P.status, 11)) break;
           const uint32_t s0 = sbase + L::kStgOff + (half * 2) * L::kStgSlab;
-          tma_store_2d(&tmY, s0, nt + half * 128, m0);
-          tma_store_2d(&tmY, s0 + L::kStgSlab, nt + half * 128 + 64, m0);
+          if (P.Mq) {
+            tma_store_2d(&tmY, s0, nt / 4 + half * 32, m0);            // 128 rows x 32 bytes of packed codes
+          } else {
+            tma_store_2d(&tmY, s0, nt + half * 128, m0);
+            tma_store_2d(&tmY, s0 + L::kStgSlab, nt + half * 128 + 64, m0);
+          }
           tma_store_commit();
           tma_store_wait_read();
           mbar_arrive(stg_empty(half));
@@ -420,6 +455,19 @@ static bool make_out_map(CUtensorMap* m, const void* base, int M, int N) {
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tensor map over the packed codes [M, N/4 bytes] the fused SwiGLU epilogue writes; one box = 128 rows x 32 bytes.
+static bool make_codes_map(CUtensorMap* m, const void* base, int M, int row_bytes) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)M};
+  const cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
+  const cuuint32_t box[2] = {32, (cuuint32_t)HR};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int NS, int NPK>
 static int launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, GemmParams P) {
   using L = Smem<NS, NPK>;
@@ -449,7 +497,9 @@ static int launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, GemmPar
   CUtensorMap tmA, tmB, tmY;
   if (!make_map(&tmA, Xq, P.M, P.K, CU_TENSOR_MAP_SWIZZLE_64B) || !make_map(&tmB, Wq, P.N, P.K, CU_TENSOR_MAP_SWIZZLE_NONE))
     return FPT_ERR_CUDA;
-  if (P.Y) { if (!make_out_map(&tmY, P.Y, P.M, P.N)) return FPT_ERR_CUDA; } else tmY = tmA;   // unused without Y
+  if (P.Mq) { if (!make_codes_map(&tmY, P.Mq, P.M, P.N / 4)) return FPT_ERR_CUDA; }
+  else if (P.Y) { if (!make_out_map(&tmY, P.Y, P.M, P.N)) return FPT_ERR_CUDA; }
+  else tmY = tmA;                                                                  // unused without an output tile
   P.tiles_m = (P.M + TM - 1) / TM;
   P.num_tiles = P.tiles_m * ((P.N + TN - 1) / TN);
   P.kblocks = P.K / BK;

@@ -113,12 +113,12 @@ extern "C" int fpt_interleave_gate_up(void* stream, const uint8_t* Wg_q, const u
                                       const void* sw_u, int scale_dtype, int d_ff, int K, uint8_t* Wgu_q,
                                       void* sw_gu) {
   if (!Wg_q || !Wu_q || !sw_g || !sw_u || !Wgu_q || !sw_gu || d_ff <= 0 || K <= 0) return FPT_ERR_BAD_ARG;
-  if (d_ff % 128 != 0 || K % 32 != 0) return FPT_ERR_UNSUPPORTED;
+  if (d_ff % 64 != 0 || K % 32 != 0) return FPT_ERR_UNSUPPORTED;
   if (scale_dtype != FPT_DTYPE_F32 && scale_dtype != FPT_DTYPE_F16) return FPT_ERR_BAD_ARG;
   cudaStream_t st = (cudaStream_t)stream;
-  const size_t row = (size_t)K / 2, grp = 128 * row;          // bytes of 128 packed rows
-  const size_t sgrp = 128 * (scale_dtype == FPT_DTYPE_F16 ? 2 : 4);
-  const size_t groups = (size_t)d_ff / 128;
+  const size_t row = (size_t)K / 2, grp = 64 * row;           // bytes of 64 packed rows
+  const size_t sgrp = 64 * (scale_dtype == FPT_DTYPE_F16 ? 2 : 4);
+  const size_t groups = (size_t)d_ff / 64;
   cudaError_t e;
   e = cudaMemcpy2DAsync(Wgu_q, 2 * grp, Wg_q, grp, grp, groups, cudaMemcpyDeviceToDevice, st);
   if (e == cudaSuccess) e = cudaMemcpy2DAsync(Wgu_q + grp, 2 * grp, Wu_q, grp, grp, groups, cudaMemcpyDeviceToDevice, st);

@@ -90,7 +90,8 @@ def _mlp_case(M, d, d_ff, seed, with_prev, residual):
 
 
 @pytest.mark.parametrize("M,d,d_ff,with_prev,residual", [(96, 256, 512, True, True), (130, 512, 1408, False, False),
-                                                         (33, 1024, 3584, True, False)])
+                                                         (33, 1024, 3584, True, False), (300, 1024, 3584, True, True),
+                                                         (513, 256, 640, False, True)])
 def test_decoder_mlp_parity(M, d, d_ff, with_prev, residual):
     Y, s_out, ref = _mlp_case(M, d, d_ff, 2, with_prev, residual)
     assert np.array_equal(host(s_out), ref["s_out"])

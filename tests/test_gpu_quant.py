@@ -86,8 +86,8 @@ def test_silu_mul_quant_bit_exact(M, K, inter):
     qp = B.QParams(4, True, 0.23, 0)
     if inter:
         gu = torch.empty((M, 2 * K), dtype=torch.bfloat16)
-        gu.view(M, K // 128, 2, 128)[:, :, 0, :] = g.view(M, K // 128, 128)
-        gu.view(M, K // 128, 2, 128)[:, :, 1, :] = u.view(M, K // 128, 128)
+        gu.view(M, K // 64, 2, 64)[:, :, 0, :] = g.view(M, K // 64, 64)
+        gu.view(M, K // 64, 2, 64)[:, :, 1, :] = u.view(M, K // 64, 64)
         xq, _ = B.fpt_act_quant(dev(gu), qp, B.SILU_MUL | B.GU_INTERLEAVED | B.SCALE_INPUT, 0.0, s_in=dev(s_n))
     else:
         xq, _ = B.fpt_act_quant(dev(g), qp, B.SILU_MUL | B.SCALE_INPUT, 0.0, X2=dev(u), s_in=dev(s_n))
@@ -122,8 +122,8 @@ def test_interleave_gate_up_layout():
     su = torch.from_numpy(rng.standard_normal(d_ff).astype(np.float32))
     wgu, sw = B.fpt_interleave_gate_up(dev(g), dev(u), dev(sg), dev(su))
     wgu, sw = host(wgu), host(sw)
-    for r in range(d_ff // 128):
-        assert np.array_equal(wgu[256 * r:256 * r + 128], g[128 * r:128 * r + 128].numpy())
-        assert np.array_equal(wgu[256 * r + 128:256 * r + 256], u[128 * r:128 * r + 128].numpy())
-        assert np.array_equal(sw[256 * r:256 * r + 128], sg[128 * r:128 * r + 128].numpy())
-        assert np.array_equal(sw[256 * r + 128:256 * r + 256], su[128 * r:128 * r + 128].numpy())
+    for r in range(d_ff // 64):
+        assert np.array_equal(wgu[128 * r:128 * r + 64], g[64 * r:64 * r + 64].numpy())
+        assert np.array_equal(wgu[128 * r + 64:128 * r + 128], u[64 * r:64 * r + 64].numpy())
+        assert np.array_equal(sw[128 * r:128 * r + 64], sg[64 * r:64 * r + 64].numpy())
+        assert np.array_equal(sw[128 * r + 64:128 * r + 128], su[64 * r:64 * r + 64].numpy())
