@@ -44,6 +44,9 @@ size_t gemm_decode_scratch_bytes(int M);
 int gemm_decode_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, const GemmParams& P, void* scratch);
 inline size_t gemm_scratch_bytes(int M) { return M <= 64 ? gemm_decode_scratch_bytes(M) : 0; }
 
+// gemm_decode_small.cu: register-only weight streaming for M <= 16 (no scratch).
+int gemm_decode_small_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, const GemmParams& P);
+
 // gemm_w4a4_2cta.cu: the CTA-pair kernel (256 x 256 tiles) behind gemm_launch for prefill sizes.
 int gemm_pair_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, const GemmParams& P);
 

@@ -331,6 +331,7 @@ static int launch_gemm(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, Ge
 }
 
 int gemm_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, const GemmParams& P) {
+  if (P.M <= 16) return gemm_decode_small_launch(st, Xq, Wq, P);
   if (P.M <= 64 && P.scratch) return gemm_decode_launch(st, Xq, Wq, P, P.scratch);
   if (P.M > 128 && P.N > 128) return gemm_pair_launch(st, Xq, Wq, P);
   if (P.N <= 64) return launch_gemm<64, 4, 4, 8>(st, Xq, Wq, P);
