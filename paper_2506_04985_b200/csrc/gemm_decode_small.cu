@@ -47,7 +47,7 @@ __device__ __forceinline__ void mma_16x8x32(int (&c)[4], uint32_t a0, uint32_t a
 }
 
 template <int NW, int NT, bool kBUnsigned>
-__global__ void __launch_bounds__(NW * 32) gemm_w4a4_decode_small_kernel(const uint8_t* __restrict__ Xq,
+__global__ void __launch_bounds__(NW * 32, 768 / (NW * 32)) gemm_w4a4_decode_small_kernel(const uint8_t* __restrict__ Xq,
                                                                           const uint8_t* __restrict__ Wq, const Params D) {
   __shared__ int part[NW][kRows][8 * NT];
   const GemmParams& P = D.g;
@@ -73,6 +73,22 @@ __global__ void __launch_bounds__(NW * 32) gemm_w4a4_decode_small_kernel(const u
   for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
     for (int j = 0; j < 4; ++j) acc[nt][j] = 0;
+  // what the epilogue needs from global memory, requested now so that it has arrived by then
+  // (thread o < 16 * 8 * NT finishes output o: weight row o % 16 of token o / 16)
+  const int o_r = threadIdx.x % kRows, o_tok = threadIdx.x / kRows;
+  const int o_n = n0 + o_r;
+  const bool o_ok = threadIdx.x < kRows * 8 * NT && o_n < P.N && o_tok < P.M;
+  float o_sw = 0.0f, o_ct = P.act_scale, o_rs = 1.0f, o_res = 0.0f;
+  int o_zw = 0;
+  if (o_ok) {
+    o_sw = load_scale(P.sw, P.scale_dtype, o_n);
+    if (P.wsum) o_zw = P.zero_point * __ldg(P.wsum + o_n);
+    if (P.post) o_ct = __fmul_rn(P.act_scale, __ldg(P.post + o_tok));
+    if (P.residual) {
+      o_res = __bfloat162float(P.residual[(size_t)o_tok * P.N + o_n]);
+      if (P.res_scale) o_rs = __ldg(P.res_scale + o_tok);
+    }
+  }
 
   constexpr int U = 4;                                   // blocks in flight per warp
   const uint4 zero = make_uint4(0, 0, 0, 0);
@@ -115,24 +131,17 @@ __global__ void __launch_bounds__(NW * 32) gemm_w4a4_decode_small_kernel(const u
   }
   __syncthreads();
   // one thread per output: consecutive threads take consecutive weight rows of one token
-  for (int o = threadIdx.x; o < kRows * 8 * NT; o += NW * 32) {
-    const int r = o % kRows, tok = o / kRows;
-    const int n = n0 + r;
-    if (n >= P.N || tok >= P.M) continue;
+  static_assert(kRows * 8 * NT <= NW * 32, "one output per thread");
+  if (o_ok) {
     int s = 0;
 #pragma unroll
-    for (int w = 0; w < NW; ++w) s += part[w][r][tok];
-    int a = s >> 8;
-    if (P.wsum) a -= P.zero_point * __ldg(P.wsum + n);
-    const size_t idx = (size_t)tok * P.N + n;
+    for (int w = 0; w < NW; ++w) s += part[w][o_r][o_tok];
+    const int a = (s >> 8) - o_zw;
+    const size_t idx = (size_t)o_tok * P.N + o_n;
     if (P.acc_out) P.acc_out[idx] = a;
     if (P.Y) {
-      const float ct = P.post ? __fmul_rn(P.act_scale, __ldg(P.post + tok)) : P.act_scale;
-      float y = __fmul_rn(__fmul_rn((float)a, load_scale(P.sw, P.scale_dtype, n)), ct);
-      if (P.residual) {
-        const float rs = P.res_scale ? __ldg(P.res_scale + tok) : 1.0f;
-        y = __fadd_rn(y, __fmul_rn(__bfloat162float(P.residual[idx]), rs));
-      }
+      float y = __fmul_rn(__fmul_rn((float)a, o_sw), o_ct);
+      if (P.residual) y = __fadd_rn(y, __fmul_rn(o_res, o_rs));
       P.Y[idx] = __float2bfloat16_rn(y);
     }
   }
