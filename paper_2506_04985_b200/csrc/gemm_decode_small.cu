@@ -12,8 +12,9 @@
 // The activations (a few KB) are read through L1 by every warp.  Warps add their partial
 // accumulators through shared memory -- integers, so the order does not matter.
 //
-// The tensor-memory kernel of gemm_decode.cu keeps the sizes from 17 to 64 tokens, where this
-// form would need too many registers and legacy-MMA issue slots.
+// The tensor-memory kernel of gemm_decode.cu keeps the sizes from 17 to 64 tokens: with four or
+// eight token groups this form was measured 1.5 to 2.5 times slower than that kernel (registers,
+// re-widening the activations per group, legacy-MMA issue rate).
 #include "fpt_internal.cuh"
 
 namespace fpt {
@@ -74,19 +75,25 @@ __global__ void __launch_bounds__(NW * 32, 768 / (NW * 32)) gemm_w4a4_decode_sma
 #pragma unroll
     for (int j = 0; j < 4; ++j) acc[nt][j] = 0;
   // what the epilogue needs from global memory, requested now so that it has arrived by then
-  // (thread o < 16 * 8 * NT finishes output o: weight row o % 16 of token o / 16)
-  const int o_r = threadIdx.x % kRows, o_tok = threadIdx.x / kRows;
-  const int o_n = n0 + o_r;
-  const bool o_ok = threadIdx.x < kRows * 8 * NT && o_n < P.N && o_tok < P.M;
-  float o_sw = 0.0f, o_ct = P.act_scale, o_rs = 1.0f, o_res = 0.0f;
-  int o_zw = 0;
-  if (o_ok) {
-    o_sw = load_scale(P.sw, P.scale_dtype, o_n);
-    if (P.wsum) o_zw = P.zero_point * __ldg(P.wsum + o_n);
-    if (P.post) o_ct = __fmul_rn(P.act_scale, __ldg(P.post + o_tok));
-    if (P.residual) {
-      o_res = __bfloat162float(P.residual[(size_t)o_tok * P.N + o_n]);
-      if (P.res_scale) o_rs = __ldg(P.res_scale + o_tok);
+  // (output o = weight row o % 16 of token o / 16; a thread finishes outputs tid, tid + blockDim, ...)
+  constexpr int kOut = kRows * 8 * NT, kPer = (kOut + NW * 32 - 1) / (NW * 32);
+  float o_sw[kPer], o_ct[kPer], o_rs[kPer], o_res[kPer];
+  int o_zw[kPer];
+  bool o_ok[kPer];
+#pragma unroll
+  for (int q = 0; q < kPer; ++q) {
+    const int o = threadIdx.x + q * NW * 32;
+    const int o_n = n0 + o % kRows, o_tok = o / kRows;
+    o_ok[q] = o < kOut && o_n < P.N && o_tok < P.M;
+    o_sw[q] = 0.0f; o_ct[q] = P.act_scale; o_rs[q] = 1.0f; o_res[q] = 0.0f; o_zw[q] = 0;
+    if (o_ok[q]) {
+      o_sw[q] = load_scale(P.sw, P.scale_dtype, o_n);
+      if (P.wsum) o_zw[q] = P.zero_point * __ldg(P.wsum + o_n);
+      if (P.post) o_ct[q] = __fmul_rn(P.act_scale, __ldg(P.post + o_tok));
+      if (P.residual) {
+        o_res[q] = __bfloat162float(P.residual[(size_t)o_tok * P.N + o_n]);
+        if (P.res_scale) o_rs[q] = __ldg(P.res_scale + o_tok);
+      }
     }
   }
 
@@ -130,18 +137,21 @@ __global__ void __launch_bounds__(NW * 32, 768 / (NW * 32)) gemm_w4a4_decode_sma
     part[warp][g + 8][nt * 8 + 2 * t + 1] = acc[nt][3];
   }
   __syncthreads();
-  // one thread per output: consecutive threads take consecutive weight rows of one token
-  static_assert(kRows * 8 * NT <= NW * 32, "one output per thread");
-  if (o_ok) {
+  // consecutive threads take consecutive weight rows of one token
+#pragma unroll
+  for (int q = 0; q < kPer; ++q) {
+    if (!o_ok[q]) continue;
+    const int o = threadIdx.x + q * NW * 32;
+    const int o_r = o % kRows, o_tok = o / kRows;
     int s = 0;
 #pragma unroll
     for (int w = 0; w < NW; ++w) s += part[w][o_r][o_tok];
-    const int a = (s >> 8) - o_zw;
-    const size_t idx = (size_t)o_tok * P.N + o_n;
+    const int a = (s >> 8) - o_zw[q];
+    const size_t idx = (size_t)o_tok * P.N + n0 + o_r;
     if (P.acc_out) P.acc_out[idx] = a;
     if (P.Y) {
-      float y = __fmul_rn(__fmul_rn((float)a, o_sw), o_ct);
-      if (P.residual) y = __fadd_rn(y, __fmul_rn(o_res, o_rs));
+      float y = __fmul_rn(__fmul_rn((float)a, o_sw[q]), o_ct[q]);
+      if (P.residual) y = __fadd_rn(y, __fmul_rn(o_res[q], o_rs[q]));
       P.Y[idx] = __float2bfloat16_rn(y);
     }
   }
@@ -162,7 +172,7 @@ int gemm_decode_small_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* 
   using namespace decode_small;
   Params D;
   D.g = P;
-  D.ntiles = P.M <= 8 ? 1 : 2;
+  D.ntiles = (P.M + 7) / 8;
   D.kblocks = P.K / 128;
   // few row strips (a short, wide matrix): more warps per strip, so that enough loads are in flight
   const bool wide = (P.N + kRows - 1) / kRows < 600;
