@@ -7,7 +7,7 @@ import torch
 from oracle import quantizers as OQ, linear as OL
 from oracle.int_matmul import int_matmul
 from oracle.epilogue import dequant_epilogue
-from paper_2506_04985_b200 import binding as B, synth
+from paper_2506_04985_b200 import binding as B, fold, synth
 from helpers import dev, host, oqp, bf16_host, assert_bf16_close
 
 pytestmark = pytest.mark.gpu
@@ -109,11 +109,31 @@ def test_config2_attention_projections_sampled():
     r = OQ.rms_reciprocal(xf[:256], 1e-5)
     qp = B.QParams(4, True, float(OQ.calibrate_static_scale(xf[:256] * r[:, None], OQ.QParams())), 0)
     xd = dev(x)
-    for name, N in (("q", 4096), ("k", 1024)):
-        w = synth.weights(N, K, 0.02, 0, "cfg2/w" + name)
+    # the mergeable transforms are folded into the weights offline, in float64, before quantisation
+    raw = {n: synth.f32(synth.weights(N, K, 0.02, 0, "cfg2/w" + n)).astype(np.float64)
+           for n, N in (("q", 4096), ("k", 1024), ("v", 1024), ("o", 4096))}
+    phi, s = synth.tk_params(8, 128, 0, "cfg2/tk")
+    fq, fk = fold.fold_pre_rope(raw["q"], raw["k"], phi, s, 8, 128, "half")
+    fv, fo = fold.fold_value(raw["v"], raw["o"], synth.tv_params(8, 128, 0, "cfg2/tv"), 8, 128)
+    folded = {"q": fq, "k": fk, "v": fv, "o": fo}
+    for name, N in (("q", 4096), ("k", 1024), ("v", 1024)):
+        w = synth.to_bf16(folded[name])
         wq, sw, _ = B.fpt_quantize_weights(dev(w))
         cw, d, _ = OQ.quantize_weights(synth.f32(w))
         Y, s_out = B.fpt_w4a4_linear(xd, wq, sw, qp, B.RMSNORM, 1e-5)
         ref = OL.w4a4_linear(xf[rows], cw, d, oqp(qp), True, False, 1e-5)
         assert np.array_equal(host(s_out)[rows], ref["s_out"])
         assert assert_bf16_close(bf16_host(Y)[rows], ref["y"], "cfg2 " + name) == 0
+    # output projection: its input is the attention output, scaled per token by S_n before the grid
+    ao = synth.activations(M, K, 0, "cfg2/ao", law="student_t3", outlier_frac=0.005, outlier_gain=50.0)
+    s_in = synth.per_token_scale(M, 0, "cfg2/s_in")
+    aof = synth.f32(ao)
+    qp_o = B.QParams(4, True, 0.75, 0)       # a grid fine enough that all 16 codes occur (the L_3 grid of
+                                             # these outlier-heavy activations uses only three of them)
+    w = synth.to_bf16(folded["o"])
+    wq, sw, _ = B.fpt_quantize_weights(dev(w))
+    cw, d, _ = OQ.quantize_weights(synth.f32(w))
+    Y, s_out = B.fpt_w4a4_linear(dev(ao), wq, sw, qp_o, B.SCALE_INPUT, 1e-5, s_in=dev(s_in))
+    ref = OL.w4a4_linear(aof[rows], cw, d, oqp(qp_o), False, True, 1e-5, s_in.numpy()[rows])
+    assert len(np.unique(ref["codes"])) >= 8
+    assert assert_bf16_close(bf16_host(Y)[rows], ref["y"], "cfg2 o") == 0
