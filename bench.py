@@ -349,6 +349,41 @@ def run_gpu(args):
                               "peak": peaks["hbm_gbs"], "unit": "GB/s",
                               "frac": aq_bytes / (kern_us["act_quant_x"] * 1e-6) / 1e9 / peaks["hbm_gbs"]}}
 
+    # ---- the other configurations, one graph-replayed measurement each (rank 0; timing does not
+    # depend on values, so operands are random codes / random bf16 made on the device) -------------
+    other = {}
+    if rank == 0 and not args.no_extras:
+        del sets, step_graphs
+        torch.cuda.empty_cache()
+        from paper_2506_04985_b200 import microbench as MB
+
+        def measure(kind, M, N, K, reps, f16=False):
+            nsets = max(2, min(8, int(300e6 / max(1.0, N * K / 2))))
+            runs, ops, nbytes = MB.make_case(kind, M, N, K, nsets, dev, f16)
+            us = MB.time_case_graph(runs, reps)
+            del runs
+            torch.cuda.empty_cache()
+            return us, ops, nbytes
+
+        us, ops, _ = measure("mlp", 4096, D_FF, HID, 10)
+        other["configs[2] SwiGLU MLP block, 4096 tokens (4 kernels)"] = {
+            "us": us, "TOP/s": ops / us / 1e6, "frac_of_int8_peak": ops / us / 1e6 / int8_peak}
+        dec = {}
+        for n, k in ((D_FF, HID), (HID, D_FF)):
+            for m in (1, 8, 32, 64):
+                us, _, nbytes = measure("gemm", m, n, k, 50, True)
+                dec[f"M={m} {k}->{n}"] = {"us": us, "GB/s": nbytes / us / 1e3, "frac_of_hbm_peak": nbytes / us / 1e3 / peaks["hbm_gbs"]}
+        other["configs[3] decode matmuls, packed weights streamed once, fp16 scales"] = dec
+        c5 = {}
+        for tokens in (512, 2048):
+            t_us, t_ops = 0.0, 0.0
+            for n, k in ((10240, 8192), (8192, 8192), (57344, 8192), (8192, 28672)):     # fused QKV, O, gate||up, down
+                us, ops, _ = measure("linear", tokens, n, k, 5)
+                t_us += us
+                t_ops += ops
+            c5[f"{tokens} tokens"] = {"us_per_layer_linears": t_us, "tokens_per_s": tokens / t_us * 1e6, "TOP/s": t_ops / t_us / 1e6}
+        other["configs[4] 70B-class layer linears (act_quant + matmul each; SwiGLU unfused)"] = c5
+
     if rank == 0:
         rows = M_TOK
         cpu_tops, cpu_dt = time_oracle(rows, 8)
@@ -364,7 +399,7 @@ def run_gpu(args):
                 "e2e": {"value": e2e_tops, "unit": "TOPS", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                         "steps": e2e_steps},
                 "gpu_launches": 4 * args.steps, "launch_mode": "one CUDA graph per step (4 kernels), replayed",
-                "clocks": clocks, "roofline": roofline, "kernel_us": kern_us,
+                "clocks": clocks, "roofline": roofline, "kernel_us": kern_us, "other_configs": other,
                 "cpu_baseline": {"value": cpu_tops, "unit": "TOPS", "cores": blas_threads(), "kind": "oracle",
                                  "sample": f"{rows} of {M_TOK} token rows x all {N_QKV + N_O} output columns, "
                                            f"8 repetitions, {cpu_dt:.2f} s each"}}
@@ -379,6 +414,7 @@ def main():
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours")
+    ap.add_argument("--no-extras", action="store_true", help="skip the one-shot measurements of the other configurations")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
