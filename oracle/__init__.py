@@ -19,6 +19,8 @@ Modules and the passages they follow
                 value transform (Sec. 3.1.2), per-token residual scaling
                 (Sec. 3.1.3), fp64 attention / MLP references used to prove
                 function preservation
+    hadamard    block-wise Hadamard transform at the down-projection input (Sec. 3.1 last
+                paragraph; App. A transform table; App. D "Hadamard non-powers of 2")
     linear      the composed entry points (one W4A4 linear; one SwiGLU MLP block)
 
 Parity status: every function is pinned by a CPU test (tests/test_oracle_*.py)

@@ -17,6 +17,7 @@ import numpy as np
 from .quantizers import QParams, act_quant, silu_mul_quant
 from .int_matmul import int_matmul
 from .epilogue import dequant_epilogue, inverse_of_pre
+from .hadamard import block_hadamard_f32
 
 F32 = np.float32
 
@@ -41,12 +42,19 @@ def w4a4_linear(x, wq, sw, qp, rmsnorm=True, scale_input=False, eps=1e-5, s_in=N
 
 
 def decoder_mlp(x, wg_q, sw_g, wu_q, sw_u, wd_q, sw_d, qp_in, qp_mid, eps=1e-5,
-                s_prev=None, add_residual=False):
-    """Returns dict(xq, g, u, m, mq, y, s_out)."""
+                s_prev=None, add_residual=False, hadamard=False):
+    """Returns dict(xq, g, u, m, mq, y, s_out).
+
+    hadamard=True inserts the online block-wise Hadamard transform at the down-projection input
+    (Sec. 3.1, last paragraph): the grid sees S_n * H(m) instead of S_n * m; `wd_q` must then be
+    the quantised down projection with the inverse transform merged into it."""
     xq, s_n, p, r = act_quant(x, qp_in, rmsnorm=True, scale_input=False, eps=eps, s_in=s_prev)
     g = dequant_epilogue(int_matmul(xq, wg_q, qp_in.z), sw_g, qp_in.scale)
     u = dequant_epilogue(int_matmul(xq, wu_q, qp_in.z), sw_u, qp_in.scale)
     mq, m = silu_mul_quant(g, u, qp_mid, s_n)
+    if hadamard:
+        h = block_hadamard_f32(m)
+        mq, _, _, _ = act_quant(h, qp_mid, rmsnorm=False, scale_input=True, s_in=s_n)
     acc_d = int_matmul(mq, wd_q, qp_mid.z)
     res = None
     if add_residual:

@@ -12,6 +12,8 @@ precision); round to the storage type afterwards.
     fold_norm_weight       RMSNorm weight gamma into the linears that read the normalised vector
     fold_up_down_scaler    Sec. 3.1 (last paragraph): per-channel scaler between up and down projection
     fold_residual_rotation Sec. 3.1 (last paragraph): one orthogonal matrix on the residual stream
+    fold_down_hadamard     Sec. 3.1 (last paragraph), App. D: inverse of the online block-wise Hadamard
+                           transform at the down-projection input, merged into the down projection
 
 Readings of the paper used here (the same as everywhere in this package): every 2x2 block of
 T_k is a proper rotation times ONE scale shared by its two coordinates; under grouped-query
@@ -99,3 +101,31 @@ def fold_residual_rotation(readers, writers, rot):
     assert np.allclose(rot @ rot.T, np.eye(rot.shape[0]), atol=1e-10), "R must be orthogonal"
     return ([np.asarray(w, dtype=np.float64) @ rot for w in readers],
             [rot.T @ np.asarray(w, dtype=np.float64) for w in writers])
+
+
+def hadamard_block_size(d):
+    """Group size of the block-wise Hadamard on d channels: the largest power of two dividing d
+    (App. D "Hadamard non-powers of 2": groups of a power-of-two size, no zero padding)."""
+    return d & (-d)
+
+
+def _fwht_last_axis(a):
+    """Unnormalised Walsh-Hadamard transform (Sylvester order) along the last axis, float64."""
+    n = a.shape[-1]
+    if n == 1:
+        return a
+    half = n // 2
+    top, bot = _fwht_last_axis(a[..., :half]), _fwht_last_axis(a[..., half:])
+    return np.concatenate([top + bot, top - bot], axis=-1)
+
+
+def fold_down_hadamard(wd, block=None):
+    """The activations entering the down projection are transformed online, group by group, with the
+    orthonormal Hadamard matrix H (fpt_decoder_mlp with mid_hadamard = 1); H is symmetric and its own
+    inverse, so the merged weight is W_d <- W_d blockdiag(H, ..., H) on the input columns."""
+    wd = np.asarray(wd, dtype=np.float64)
+    d = wd.shape[1]
+    block = block or hadamard_block_size(d)
+    assert d % block == 0 and block & (block - 1) == 0
+    g = wd.reshape(wd.shape[0], d // block, block)
+    return (_fwht_last_axis(g) / np.sqrt(block)).reshape(wd.shape[0], d)

@@ -4,6 +4,7 @@ against the float64 reference model: merged and unmerged networks must compute t
 import numpy as np
 import pytest
 
+from oracle import hadamard as OH
 from oracle import transforms as OT
 from paper_2506_04985_b200 import fold, synth
 
@@ -90,3 +91,21 @@ def test_residual_rotation_keeps_a_two_block_network():
     assert _rel(got, ref @ rot) < 1e-10
     with pytest.raises(AssertionError):
         fold.fold_residual_rotation([layers[0][0]], [layers[0][2]], rot * 1.01)
+
+
+@pytest.mark.parametrize("dff", [96, 224, 1024])
+def test_down_hadamard_fold_matches_the_definition_and_keeps_the_mlp(dff):
+    rng = np.random.default_rng(8)
+    d, L = 40, 6
+    wg, wu, wd = (rng.standard_normal(s) * 0.2 for s in ((dff, d), (dff, d), (d, dff)))
+    hb = OH.block_hadamard_matrix(dff)
+    assert fold.hadamard_block_size(dff) == OH.largest_pow2_divisor(dff)
+    wd2 = fold.fold_down_hadamard(wd)
+    assert np.allclose(wd2, wd @ hb, rtol=1e-12, atol=1e-13)
+    # the network with the online transform in front of the merged weight computes the same function
+    xn = rng.standard_normal((L, d))
+    g = xn @ wg.T
+    m = g / (1.0 + np.exp(-g)) * (xn @ wu.T)
+    ref = m @ wd.T
+    got = (m @ hb.T) @ wd2.T
+    assert _rel(got, ref) < 1e-10
