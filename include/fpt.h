@@ -147,6 +147,24 @@ int fpt_act_quant(void* stream, const void* X, int M, int K, int ldx,
                   const void* X2, const float* s_in, uint8_t* Xq, float* s_out);
 
 /*
+ * Online block-wise Hadamard transform + per-token scale + static quantise + pack, for the input of
+ * the down projection (Sec. 3.1, last paragraph; App. A transform table: H_n = n^(-1/2) (x) [[1,1],[1,-1]];
+ * App. D "Hadamard non-powers of 2").  The K channels are split into K / B groups of
+ * B = largest power of two dividing K (256 <= B <= 4096), each group is multiplied by H_B; there is no
+ * zero padding.  Per token t:
+ *   m_tk = X[t,k]                    (FPT_SILU_MUL | FPT_GU_INTERLEAVED: bf16(silu(g) * u) from the
+ *                                     64-column gate||up layout, X is [M, 2K])
+ *   h    = H_B applied group-wise, float32 butterflies (a, b) -> (a + b, a - b) with partner distance
+ *          1, 2, 4, ..., B/2 in this order, then one multiply by float32(B^(-1/2))
+ *   q_tk = clamp(rne((h_tk * p_t) * (1/D)) + z),  p_t = s_in[t] with FPT_SCALE_INPUT, else 1
+ * The weight that consumes the codes must have the inverse transform merged into its input columns
+ * (W <- W blockdiag(H_B); H_B is symmetric and orthogonal).
+ *   X [M, ldx] bf16;  Xq [M, K/2] packed codes out;  K % 256 == 0.
+ */
+int fpt_hadamard_quant(void* stream, const void* X, int M, int K, int ldx,
+                       const fpt_qparams* qp, int flags, const float* s_in, uint8_t* Xq);
+
+/*
  * Steps (2)+(3) on already packed operands (App. J "Setup"; App. B "Static quantization"):
  *   acc[t,n] = sum_k (qa[t,k] - z) * qw[n,k]                 exact int32
  *   y[t,n]   = bf16( ((float)acc * sw[n]) * c_t  [+ res[t,n] * res_scale[t]] )
@@ -217,6 +235,8 @@ int fpt_w4a4_linear_static(void* stream, const void* X, int M, int K,
  *   g, u = W4A4 linears of X~ (bf16)                          grid qp_in
  *   m = bf16(silu(g) * u);  quantise m * S_n                  grid qp_mid (scaler at the
  *                                                              down-projection input)
+ *        with mid_hadamard = 1 the grid sees S_n * H(m) (fpt_hadamard_quant) and Wd_q must be the
+ *        quantised W_d blockdiag(H) (Sec. 3.1 last paragraph: the one online transform)
  *   Y~ = W4A4 down projection  (= S_n * Y_n, Eq. 5)
  *   Y  = bf16(Y~ + X * r)  if add_residual  (Z~_n = X~_n + Y~_n)   else bf16(Y~)
  *   Wgu_q [2 d_ff, d/2] and sw_gu [2 d_ff] in the layout of fpt_interleave_gate_up;
@@ -227,7 +247,7 @@ int fpt_w4a4_linear_static(void* stream, const void* X, int M, int K,
 int fpt_decoder_mlp(void* stream, const void* X, int M, int d, int d_ff,
                     const uint8_t* Wgu_q, const void* sw_gu, const uint8_t* Wd_q, const void* sw_d,
                     int scale_dtype, const fpt_qparams* qp_in, const fpt_qparams* qp_mid, float eps,
-                    const float* s_prev, float* s_out, int add_residual,
+                    const float* s_prev, float* s_out, int add_residual, int mid_hadamard,
                     void* Y, void* workspace, size_t workspace_bytes);
 
 /* Bytes of caller-provided scratch an entry point needs (op = FPT_OP_*).

@@ -21,7 +21,7 @@ RMSNORM, SCALE_INPUT, SILU_MUL, GU_INTERLEAVED = 1, 2, 4, 8
 POST_NONE, POST_INVERSE_OF_PRE, POST_VECTOR = 0, 1, 2
 OP_LINEAR, OP_MLP, OP_GEMM = 0, 1, 2
 
-EXPORTS = ["fpt_version", "fpt_strerror", "fpt_quantize_weights", "fpt_interleave_gate_up", "fpt_act_quant",
+EXPORTS = ["fpt_version", "fpt_strerror", "fpt_quantize_weights", "fpt_interleave_gate_up", "fpt_act_quant", "fpt_hadamard_quant",
            "fpt_w4a4_gemm", "fpt_w4a4_linear", "fpt_w4a4_linear_static", "fpt_decoder_mlp", "fpt_workspace_bytes", "fpt_reset_status",
            "fpt_check_status"]
 
@@ -62,7 +62,8 @@ def lib():
         L.fpt_w4a4_gemm.argtypes = [vp, vp, vp, ci, ci, ci, vp, ci, vp, cf, ci, ci, vp, vp, vp, vp, vp, vp, sz]
         L.fpt_w4a4_linear.argtypes = [vp, vp, ci, ci, vp, vp, ci, vp, ci, qp, ci, cf, vp, ci, vp, vp, vp, vp, sz]
         L.fpt_w4a4_linear_static.argtypes = [vp, vp, ci, ci, vp, vp, ci, vp, ci, qp, ci, cf, vp, ci, vp, vp, vp]
-        L.fpt_decoder_mlp.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp, vp, ci, qp, qp, cf, vp, vp, ci, vp, vp, sz]
+        L.fpt_decoder_mlp.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp, vp, ci, qp, qp, cf, vp, vp, ci, ci, vp, vp, sz]
+        L.fpt_hadamard_quant.argtypes = [vp, vp, ci, ci, ci, qp, ci, vp, vp]
         L.fpt_workspace_bytes.restype = sz
         L.fpt_workspace_bytes.argtypes = [ci, ci, ci, ci]
         L.fpt_reset_status.argtypes = [vp, vp]
@@ -200,8 +201,19 @@ def fpt_w4a4_linear_static(X, Wq, sw, qp, flags=RMSNORM, eps=1e-5, s_in=None, po
     return Y, s_out
 
 
+def fpt_hadamard_quant(X, qp, flags=SCALE_INPUT, s_in=None, K=None, out=None):
+    """X [M, ldx] bf16 (products, or gate||up with SILU_MUL | GU_INTERLEAVED) -> Xq uint8 [M, K/2]."""
+    M, ldx = X.shape
+    if K is None:
+        K = ldx // 2 if (flags & GU_INTERLEAVED) else ldx
+    Xq = out if out is not None else torch.empty((M, K // 2), dtype=torch.uint8, device=X.device)
+    _check(lib().fpt_hadamard_quant(_stream(), _ptr(X), M, K, ldx, ctypes.byref(qp), flags, _ptr(s_in), _ptr(Xq)),
+           "fpt_hadamard_quant")
+    return Xq
+
+
 def fpt_decoder_mlp(X, Wgu_q, sw_gu, Wd_q, sw_d, qp_in, qp_mid, eps=1e-5, s_prev=None, add_residual=False,
-                    want_s_out=True, ws=None, Y=None):
+                    want_s_out=True, ws=None, Y=None, mid_hadamard=False):
     """One SwiGLU MLP block -> (Y bf16 [M, d], s_out f32 [M] or None)."""
     M, d = X.shape
     d_ff = Wgu_q.shape[0] // 2
@@ -212,6 +224,7 @@ def fpt_decoder_mlp(X, Wgu_q, sw_gu, Wd_q, sw_d, qp_in, qp_mid, eps=1e-5, s_prev
     s_out = torch.empty((M,), dtype=torch.float32, device=X.device) if want_s_out else None
     _check(lib().fpt_decoder_mlp(_stream(), _ptr(X), M, d, d_ff, _ptr(Wgu_q), _ptr(sw_gu), _ptr(Wd_q), _ptr(sw_d),
                                  _scale_dtype(sw_gu), ctypes.byref(qp_in), ctypes.byref(qp_mid), eps, _ptr(s_prev),
-                                 _ptr(s_out), int(bool(add_residual)), _ptr(Y), _ptr(ws), ws.numel()),
+                                 _ptr(s_out), int(bool(add_residual)), int(bool(mid_hadamard)), _ptr(Y), _ptr(ws),
+                                 ws.numel()),
            "fpt_decoder_mlp")
     return Y, s_out

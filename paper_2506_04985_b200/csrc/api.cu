@@ -134,7 +134,8 @@ extern "C" int fpt_w4a4_linear(void* stream, const void* X, int M, int K, const 
 extern "C" int fpt_decoder_mlp(void* stream, const void* X, int M, int d, int d_ff, const uint8_t* Wgu_q,
                                const void* sw_gu, const uint8_t* Wd_q, const void* sw_d, int scale_dtype,
                                const fpt_qparams* qp_in, const fpt_qparams* qp_mid, float eps, const float* s_prev,
-                               float* s_out, int add_residual, void* Y, void* workspace, size_t workspace_bytes) {
+                               float* s_out, int add_residual, int mid_hadamard, void* Y, void* workspace,
+                               size_t workspace_bytes) {
   if (!X || !Wgu_q || !sw_gu || !Wd_q || !sw_d || !Y) return FPT_ERR_BAD_ARG;
   int rc = check_qp(qp_in);
   if (rc) return rc;
@@ -144,6 +145,7 @@ extern "C" int fpt_decoder_mlp(void* stream, const void* X, int M, int d, int d_
   if (M <= 0 || d <= 0 || d_ff <= 0) return FPT_ERR_BAD_ARG;
   if (d % 128 != 0 || d_ff % 128 != 0 || d_ff > 32768 || d > 65535) return FPT_ERR_UNSUPPORTED;
   if (scale_dtype != FPT_DTYPE_F32 && scale_dtype != FPT_DTYPE_F16) return FPT_ERR_BAD_ARG;
+  if (mid_hadamard && (hadamard_block(d_ff) < 256 || hadamard_block(d_ff) > 4096)) return FPT_ERR_UNSUPPORTED;
   if (((uintptr_t)X | (uintptr_t)Wgu_q | (uintptr_t)Wd_q | (uintptr_t)Y | (uintptr_t)workspace) & 15)
     return FPT_ERR_ALIGNMENT;
   if (!workspace || workspace_bytes < fpt_workspace_bytes(FPT_OP_MLP, M, d_ff, d)) return FPT_ERR_WORKSPACE;
@@ -168,13 +170,26 @@ extern "C" int fpt_decoder_mlp(void* stream, const void* X, int M, int d, int d_
     P.M = M; P.N = 2 * d_ff; P.K = d;
     P.sw = sw_gu; P.scale_dtype = scale_dtype;
     P.act_scale = qp_in->scale;
-    P.Mq = Mq; P.mid_scale = sn;
-    P.mid_inv_delta = 1.0f / qp_mid->scale;
-    P.mid_qmax_minus_z = 7; P.mid_flip = 0x77777777u;
+    if (mid_hadamard) {          // the products leave as bf16 [M, d_ff]; the transform needs whole rows of them
+      P.swiglu_bf16 = 1;
+      P.Y = reinterpret_cast<__nv_bfloat16*>(GU);
+    } else {
+      P.Mq = Mq; P.mid_scale = sn;
+      P.mid_inv_delta = 1.0f / qp_mid->scale;
+      P.mid_qmax_minus_z = 7; P.mid_flip = 0x77777777u;
+    }
     P.status = reinterpret_cast<uint32_t*>(workspace);
     P.scratch = ws + kStatusBytes;
     rc = gemm_pair_launch(st, Xq, Wgu_q, P);
     if (rc) return rc;
+    if (mid_hadamard &&
+        hadamard_quant_launch(st, GU, M, d_ff, d_ff, qp_mid, 0, sn, Mq) != cudaSuccess)
+      return FPT_ERR_CUDA;
+  } else if (mid_hadamard) {
+    rc = fpt_w4a4_gemm(stream, Xq, Wgu_q, M, 2 * d_ff, d, sw_gu, scale_dtype, nullptr, qp_in->scale, 1, 0, nullptr,
+                       nullptr, nullptr, GU, nullptr, workspace, gemm_ws);
+    if (rc) return rc;
+    if (hadamard_quant_launch(st, GU, M, d_ff, 2 * d_ff, qp_mid, 1, sn, Mq) != cudaSuccess) return FPT_ERR_CUDA;
   } else {
     // gate || up in one matmul over the interleaved weight
     rc = fpt_w4a4_gemm(stream, Xq, Wgu_q, M, 2 * d_ff, d, sw_gu, scale_dtype, nullptr, qp_in->scale, 1, 0, nullptr,

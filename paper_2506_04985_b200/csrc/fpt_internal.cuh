@@ -22,6 +22,7 @@ struct GemmParams {
   // SwiGLU + quantise fused into the epilogue (gate||up matmul of the MLP block, CTA-pair kernel
   // only): with Mq set, the columns are 64 gate | 64 up | ... output features, no bf16 tile is
   // written, and m = bf16(silu(g) * u) is quantised with the per-token multiplier mid_scale[t]
+  int swiglu_bf16;             // with Y set and Mq null: Y [M, N/2] receives m itself (bf16), nothing is quantised
   uint8_t* Mq;                 // [M, N/4] packed codes of the N/2 products, or nullptr
   const float* mid_scale;      // [M] S_n
   float mid_inv_delta;         // 1/D of the grid at the down-projection input
@@ -35,6 +36,11 @@ struct GemmParams {
 cudaError_t act_quant_launch(cudaStream_t st, const void* X, int M, int K, int ldx, const fpt_qparams* qp,
                              int flags, float eps, const void* X2, const float* s_in, uint8_t* Xq,
                              float* s_out, float* post_inv, float* r_out);
+
+// hadamard_quant.cu: block-wise Hadamard + per-token scale + quantise (validated arguments only).
+int hadamard_block(int K);
+cudaError_t hadamard_quant_launch(cudaStream_t st, const void* X, int M, int K, int ldx, const fpt_qparams* qp,
+                                  int silu_inter, const float* s_in, uint8_t* Xq);
 
 // gemm_w4a4.cu: validated arguments only; returns an FPT_* code.
 int gemm_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, const GemmParams& P);

@@ -305,7 +305,7 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
-      if (P.Mq) {
+      if (P.Mq || P.swiglu_bf16) {
         // v[0..63]: gate accumulators of 64 features, v[64..127]: their up accumulators.
         // g, u = bf16 outputs of the two linears; m = bf16(silu(g) * u); code = grid(m * S_n).
         const QuantConsts qc = quant_consts(sn, P.mid_inv_delta, P.mid_qmax_minus_z, P.mid_flip);
@@ -327,11 +327,18 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             }
             mw[jj] = silu_mul_pair(gw, uw);
           }
-          codes[j8] = quant_word(make_uint4(mw[0], mw[1], mw[2], mw[3]), qc);
+          if (P.Mq) {
+            codes[j8] = quant_word(make_uint4(mw[0], mw[1], mw[2], mw[3]), qc);
+          } else {                                         // the products themselves: 128-byte rows, 128-byte swizzle
+            uint8_t* slab = smem + L::kStgOff + (half * 2) * L::kStgSlab + r * 128;
+            *reinterpret_cast<uint4*>(slab + ((j8 ^ (r & 7)) << 4)) = make_uint4(mw[0], mw[1], mw[2], mw[3]);
+          }
         }
-        uint4* stg = reinterpret_cast<uint4*>(smem + L::kStgOff + (half * 2) * L::kStgSlab + r * 32);
-        stg[0] = make_uint4(codes[0], codes[1], codes[2], codes[3]);
-        stg[1] = make_uint4(codes[4], codes[5], codes[6], codes[7]);
+        if (P.Mq) {
+          uint4* stg = reinterpret_cast<uint4*>(smem + L::kStgOff + (half * 2) * L::kStgSlab + r * 32);
+          stg[0] = make_uint4(codes[0], codes[1], codes[2], codes[3]);
+          stg[1] = make_uint4(codes[4], codes[5], codes[6], codes[7]);
+        }
       } else {
 #pragma unroll
       for (int ch = 0; ch < 4; ++ch) {
@@ -384,6 +391,8 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
           const uint32_t s0 = sbase + L::kStgOff + (half * 2) * L::kStgSlab;
           if (P.Mq) {
             tma_store_2d(&tmY, s0, nt / 4 + half * 32, m0);            // 128 rows x 32 bytes of packed codes
+          } else if (P.swiglu_bf16) {
+            tma_store_2d(&tmY, s0, nt / 2 + half * 64, m0);            // 128 rows x 64 products
           } else {
             tma_store_2d(&tmY, s0, nt + half * 128, m0);
             tma_store_2d(&tmY, s0 + L::kStgSlab, nt + half * 128 + 64, m0);
@@ -498,7 +507,7 @@ static int launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, GemmPar
   if (!make_map(&tmA, Xq, P.M, P.K, CU_TENSOR_MAP_SWIZZLE_64B) || !make_map(&tmB, Wq, P.N, P.K, CU_TENSOR_MAP_SWIZZLE_NONE))
     return FPT_ERR_CUDA;
   if (P.Mq) { if (!make_codes_map(&tmY, P.Mq, P.M, P.N / 4)) return FPT_ERR_CUDA; }
-  else if (P.Y) { if (!make_out_map(&tmY, P.Y, P.M, P.N)) return FPT_ERR_CUDA; }
+  else if (P.Y) { if (!make_out_map(&tmY, P.Y, P.M, P.swiglu_bf16 ? P.N / 2 : P.N)) return FPT_ERR_CUDA; }
   else tmY = tmA;                                                                  // unused without an output tile
   P.tiles_m = (P.M + TM - 1) / TM;
   P.num_tiles = P.tiles_m * ((P.N + TN - 1) / TN);

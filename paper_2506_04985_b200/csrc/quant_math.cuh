@@ -93,6 +93,24 @@ __device__ __forceinline__ uint32_t quant_pair(uint32_t w, const QuantConsts& c,
   return (prev * 16u + c1) * 16u + c0;
 }
 
+// The same for two float32 values (no 16-bit rounding in front of the grid).
+__device__ __forceinline__ uint32_t quant_pair_f32(float x0, float x1, const QuantConsts& c, uint32_t prev) {
+  float v0, v1;
+  unpack_f32x2(add_f32x2(mul_f32x2(mul_f32x2(pack_f32x2(x0, x1), c.np2), c.d2), c.m2), v0, v1);
+  const uint32_t c0 = (uint32_t)__viaddmin_s32_relu(max(__float_as_int(v0), 0), c.bias, 15);
+  const uint32_t c1 = (uint32_t)__viaddmin_s32_relu(max(__float_as_int(v1), 0), c.bias, 15);
+  return (prev * 16u + c1) * 16u + c0;
+}
+
+// Eight float32 values -> eight packed codes (value 0 in bits 0-3).
+__device__ __forceinline__ uint32_t quant_word_f32(const float (&x)[8], const QuantConsts& c) {
+  uint32_t w = quant_pair_f32(x[6], x[7], c, 0u);
+  w = quant_pair_f32(x[4], x[5], c, w);
+  w = quant_pair_f32(x[2], x[3], c, w);
+  w = quant_pair_f32(x[0], x[1], c, w);
+  return w ^ c.flip;
+}
+
 __device__ __forceinline__ uint32_t quant_word(const uint4& v, const QuantConsts& c) {
   uint32_t w = quant_pair(v.w, c, 0u);
   w = quant_pair(v.z, c, w);

@@ -81,7 +81,7 @@ def test_argument_errors_are_reported_before_any_launch(B):
                                B.RANGE_MINMAX, 3.0, B.DTYPE_F32, fake, fake, None)
     assert r == B.ERR_UNSUPPORTED                      # weights use the symmetric grid
     r = L.fpt_decoder_mlp(None, fake, 8, 100, 256, fake, fake, fake, fake, B.DTYPE_F32, ctypes.byref(qp),
-                          ctypes.byref(qp), 1e-5, None, None, 0, fake, fake, 1 << 30)
+                          ctypes.byref(qp), 1e-5, None, None, 0, 0, fake, fake, 1 << 30)
     assert r == B.ERR_UNSUPPORTED
     assert L.fpt_check_status(None, None) == B.ERR_BAD_ARG
 
