@@ -81,7 +81,9 @@ __device__ __forceinline__ void load_scales8(const void* sw, int scale_dtype, in
   }
 }
 
-template <int NS, int NPK>
+// kFuse: 0 plain scale-factor epilogue; 1 SwiGLU product + quantiser (codes out); 2 SwiGLU product
+// (bf16 out).  Separate instantiations keep the plain epilogue's register budget free of the others.
+template <int NS, int NPK, int kFuse>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                       const __grid_constant__ CUtensorMap tmY, const GemmParams P) {
@@ -118,7 +120,7 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     fence_mbar_init();
     prefetch_tmap(&tmA);
     prefetch_tmap(&tmB);
-    if (P.Y || P.Mq) prefetch_tmap(&tmY);
+    if (P.Y || kFuse == 1) prefetch_tmap(&tmY);
   }
   if (warp == 1) {
     tmem_alloc_pair(sbase + L::kMiscOff, kTmemCols);
@@ -283,12 +285,12 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
       float c = P.act_scale, rs = 1.0f;
       if (row_ok && P.post) c = __fmul_rn(P.act_scale, __ldg(P.post + row));
       if (row_ok && P.res_scale) rs = __ldg(P.res_scale + row);
-      const float sn = (P.Mq && row_ok) ? __ldg(P.mid_scale + row) : 0.0f;
+      const float sn = (kFuse == 1 && row_ok) ? __ldg(P.mid_scale + row) : 0.0f;
       __syncwarp();
       if (lane == 0) mbar_arrive(sc_full(b));
       if (!mbar_wait(sc_full(b), bph, abort_flag, P.status, 9)) break;
       // the staging half must have been read by the TMA store of the previous tile
-      if ((P.Y || P.Mq) && !mbar_wait(stg_empty(half), (it & 1) ^ 1u, abort_flag, P.status, 10)) break;
+      if ((P.Y || kFuse == 1) && !mbar_wait(stg_empty(half), (it & 1) ^ 1u, abort_flag, P.status, 10)) break;
       if (!mbar_wait(acc_full, it & 1, abort_flag, P.status, 4)) break;
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + half * 128;
@@ -305,7 +307,7 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
-      if (P.Mq || P.swiglu_bf16) {
+      if constexpr (kFuse != 0) {
         // v[0..63]: gate accumulators of 64 features, v[64..127]: their up accumulators.
         // g, u = bf16 outputs of the two linears; m = bf16(silu(g) * u); code = grid(m * S_n).
         const QuantConsts qc = quant_consts(sn, P.mid_inv_delta, P.mid_qmax_minus_z, P.mid_flip);
@@ -327,14 +329,14 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             }
             mw[jj] = silu_mul_pair(gw, uw);
           }
-          if (P.Mq) {
+          if constexpr (kFuse == 1) {
             codes[j8] = quant_word(make_uint4(mw[0], mw[1], mw[2], mw[3]), qc);
           } else {                                         // the products themselves: 128-byte rows, 128-byte swizzle
             uint8_t* slab = smem + L::kStgOff + (half * 2) * L::kStgSlab + r * 128;
             *reinterpret_cast<uint4*>(slab + ((j8 ^ (r & 7)) << 4)) = make_uint4(mw[0], mw[1], mw[2], mw[3]);
           }
         }
-        if (P.Mq) {
+        if constexpr (kFuse == 1) {
           uint4* stg = reinterpret_cast<uint4*>(smem + L::kStgOff + (half * 2) * L::kStgSlab + r * 32);
           stg[0] = make_uint4(codes[0], codes[1], codes[2], codes[3]);
           stg[1] = make_uint4(codes[4], codes[5], codes[6], codes[7]);
@@ -382,16 +384,16 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         }
       }
       }
-      if (P.Y || P.Mq) {
+      if (P.Y || kFuse == 1) {
         fence_proxy_async_smem();                        // staged tile -> visible to the TMA engine
         __syncwarp();
         if (lane == 0) mbar_arrive(stg_full(half));
         if (issuer) {
           if (!mbar_wait(stg_full(half), it & 1, abort_flag, P.status, 11)) break;
           const uint32_t s0 = sbase + L::kStgOff + (half * 2) * L::kStgSlab;
-          if (P.Mq) {
+          if constexpr (kFuse == 1) {
             tma_store_2d(&tmY, s0, nt / 4 + half * 32, m0);            // 128 rows x 32 bytes of packed codes
-          } else if (P.swiglu_bf16) {
+          } else if constexpr (kFuse == 2) {
             tma_store_2d(&tmY, s0, nt / 2 + half * 64, m0);            // 128 rows x 64 products
           } else {
             tma_store_2d(&tmY, s0, nt + half * 128, m0);
@@ -477,10 +479,10 @@ static bool make_codes_map(CUtensorMap* m, const void* base, int M, int row_byte
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int NS, int NPK>
+template <int NS, int NPK, int kFuse>
 static int launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, GemmParams P) {
   using L = Smem<NS, NPK>;
-  auto kern = gemm_w4a4_pair_kernel<NS, NPK>;
+  auto kern = gemm_w4a4_pair_kernel<NS, NPK, kFuse>;
   static int max_pairs = 0;                 // co-resident CTA pairs on this device
   if (!max_pairs) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kAlloc) != cudaSuccess)
@@ -520,7 +522,9 @@ static int launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, GemmPar
 }  // namespace pair
 
 int gemm_pair_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, const GemmParams& P) {
-  return pair::launch<4, 5>(st, Xq, Wq, P);
+  if (P.Mq) return pair::launch<4, 5, 1>(st, Xq, Wq, P);
+  if (P.swiglu_bf16) return pair::launch<4, 5, 2>(st, Xq, Wq, P);
+  return pair::launch<4, 5, 0>(st, Xq, Wq, P);
 }
 
 }  // namespace fpt

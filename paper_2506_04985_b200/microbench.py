@@ -4,7 +4,8 @@
     python -m paper_2506_04985_b200.microbench act_quant --M 2048 --K 4096
     python -m paper_2506_04985_b200.microbench silu_quant --M 4096 --K 14336
     python -m paper_2506_04985_b200.microbench linear    --M 64 --N 14336 --K 4096
-    python -m paper_2506_04985_b200.microbench mlp       --M 4096 --K 4096 --N 14336
+    python -m paper_2506_04985_b200.microbench hadamard_quant --M 4096 --K 14336
+    python -m paper_2506_04985_b200.microbench mlp       --M 4096 --K 4096 --N 14336      (mlp_hadamard: with the online transform)
 
 Operands are random packed codes / random bf16 values made on the device (timing does
 not depend on the values).  `--sets S` rotates S independent operand sets so that every
@@ -58,6 +59,13 @@ def make_case(kind, M, N, K, sets, dev, f16_scales=False):
             runs.append(lambda gu=gu, s=s, out=out: B.fpt_act_quant(
                 gu, qp, B.SILU_MUL | B.GU_INTERLEAVED | B.SCALE_INPUT, 0.0, s_in=s, K=K, want_s_out=False, out=out))
         return runs, 0.0, 4.5 * M * K + 4.0 * M
+    if kind == "hadamard_quant":            # products m [M, K] bf16 -> block Hadamard -> codes
+        for _ in range(sets):
+            m = _bf16(M, K, dev)
+            s = torch.rand((M,), device=dev) + 0.5
+            out = torch.empty((M, K // 2), dtype=torch.uint8, device=dev)
+            runs.append(lambda m=m, s=s, out=out: B.fpt_hadamard_quant(m, qp, B.SCALE_INPUT, s_in=s, out=out))
+        return runs, 0.0, 2.5 * M * K + 4.0 * M
     if kind == "linear":
         for _ in range(sets):
             x, wq = _bf16(M, K, dev), _codes(N, K // 2, dev)
@@ -67,7 +75,7 @@ def make_case(kind, M, N, K, sets, dev, f16_scales=False):
             runs.append(lambda x=x, wq=wq, sw=sw, y=y, ws=ws: B.fpt_w4a4_linear(
                 x, wq, sw, qp, B.RMSNORM, 1e-5, want_s_out=False, ws=ws, Y=y))
         return runs, 2.0 * M * N * K, 2.0 * M * K + N * K / 2 + N * ssz + 2.0 * M * N
-    if kind == "mlp":                      # K = d, N = d_ff
+    if kind in ("mlp", "mlp_hadamard"):    # K = d, N = d_ff
         d, dff = K, N
         for _ in range(sets):
             x = _bf16(M, d, dev)
@@ -77,7 +85,7 @@ def make_case(kind, M, N, K, sets, dev, f16_scales=False):
             y = torch.empty((M, d), dtype=torch.bfloat16, device=dev)
             ws = B.new_workspace(B.OP_MLP, M, dff, d, dev)
             runs.append(lambda x=x, wgu=wgu, sgu=sgu, wd=wd, sd=sd, y=y, ws=ws: B.fpt_decoder_mlp(
-                x, wgu, sgu, wd, sd, qp, qp, 1e-5, want_s_out=False, ws=ws, Y=y))
+                x, wgu, sgu, wd, sd, qp, qp, 1e-5, want_s_out=False, ws=ws, Y=y, mid_hadamard=kind == "mlp_hadamard"))
         return runs, 6.0 * M * d * dff, 4.0 * M * d + 1.5 * d * dff + 3 * dff * ssz
     raise ValueError(kind)
 
@@ -118,7 +126,7 @@ def time_case_graph(runs, reps, warmup=3, replays=5):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("kind", choices=["gemm", "act_quant", "silu_quant", "linear", "mlp"])
+    ap.add_argument("kind", choices=["gemm", "act_quant", "silu_quant", "hadamard_quant", "linear", "mlp", "mlp_hadamard"])
     ap.add_argument("--M", type=int, default=2048)
     ap.add_argument("--N", type=int, default=4096)
     ap.add_argument("--K", type=int, default=4096)
