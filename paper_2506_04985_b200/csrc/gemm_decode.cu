@@ -196,8 +196,6 @@ gemm_w4a4_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
       uint4 c[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) if (i < per_thread) c[i] = src[i * 64 + ctid];
-      __syncwarp();
-      if (lane == 0) mbar_arrive(pk_empty(ps));
       if (!mbar_wait(op_empty(s), ph ^ 1u, abort_flag, P.status, 8)) break;
       uint8_t* dst = smem + L::kB8Off + s * L::kB8Stage;
 #pragma unroll
@@ -212,9 +210,13 @@ gemm_w4a4_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
           *reinterpret_cast<uint4*>(rowp + (((2 * ch + 1) ^ (r & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
         }
       }
+      // One fence for both hand-overs: the widened tile becomes visible to the tensor core's async
+      // proxy, and the reads of the packed tile -- consumed by the stores above -- are ordered before
+      // the TMA write that re-fills it.  (A packed tile handed back right after its loads, before
+      // anything depends on them, can be overwritten while the loads are still in flight.)
       fence_proxy_async_smem();
       __syncwarp();
-      if (lane == 0) mbar_arrive(op_full(s));
+      if (lane == 0) { mbar_arrive(pk_empty(ps)); mbar_arrive(op_full(s)); }
       if (++ps == NPK) { ps = 0; pph ^= 1u; }
       if (++s == NS) { s = 0; ph ^= 1u; }
     }
@@ -236,8 +238,6 @@ gemm_w4a4_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
       uint32_t v[64];
 #pragma unroll
       for (int j = 0; j < 8; ++j) widen(c[j], v + 8 * j);
-      __syncwarp();
-      if (lane == 0) mbar_arrive(pk_empty(ps));
       if (!mbar_wait(op_empty(s), ph ^ 1u, abort_flag, P.status, 6)) break;
       tc_fence_after();
       const uint32_t a_tmem = tmem_base + ((uint32_t)(quad * 32) << 16) + kAStage0 + s * (BK / 4);
@@ -245,8 +245,9 @@ gemm_w4a4_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
       tmem_st_32x32(a_tmem + 32, v + 32);
       tmem_wait_st();
       tc_fence_before();
+      fence_proxy_async_smem();      // reads of the packed tile (consumed above) before the TMA write that re-fills it
       __syncwarp();
-      if (lane == 0) mbar_arrive(op_full(s));
+      if (lane == 0) { mbar_arrive(pk_empty(ps)); mbar_arrive(op_full(s)); }
     }
   } else {
     // ------------------------------------------------------------------ epilogue

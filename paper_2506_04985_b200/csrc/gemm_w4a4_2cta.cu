@@ -209,15 +209,18 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         uint32_t v[32];
 #pragma unroll
         for (int j = 0; j < 4; ++j) widen(c[j], v + 8 * j);
-        __syncwarp();
-        if (lane == 0) mbar_arrive(pk_empty(ps));
         if (!mbar_wait(op_empty(s), ph ^ 1u, abort_flag, P.status, 6)) { ok = false; break; }
         tc_fence_after();
         tmem_st_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + kAccCols + s * kAStageCols, v);
         tmem_wait_st();
         tc_fence_before();
+        // The packed tile goes back to TMA only here: its reads have been consumed (the store above
+        // depends on them) and are fenced against the async proxy, which will overwrite the tile.
+        // Handing it back right after the loads, with nothing depending on them yet, let the next
+        // TMA write overtake reads still in flight (seen as wrong weight rows, rarely, under load).
+        fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) mbar_arrive_cluster(op_full_leader + 8u * s);
+        if (lane == 0) { mbar_arrive(pk_empty(ps)); mbar_arrive_cluster(op_full_leader + 8u * s); }
         if (++ps == NPK) { ps = 0; pph ^= 1u; }
         if (++s == NS) { s = 0; ph ^= 1u; }
       }
@@ -236,8 +239,6 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         uint4 c[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) c[i] = src[i * 128 + ctid];
-        __syncwarp();
-        if (lane == 0) mbar_arrive(pk_empty(ps));
         if (!mbar_wait(op_empty(s), ph ^ 1u, abort_flag, P.status, 8)) { ok = false; break; }
         uint8_t* dst = smem + L::kB8Off + s * L::kB8Stage;
 #pragma unroll
@@ -250,9 +251,12 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
           *reinterpret_cast<uint4*>(rowp + (((2 * ch) ^ (r & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
           *reinterpret_cast<uint4*>(rowp + (((2 * ch + 1) ^ (r & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
         }
-        fence_proxy_async_smem();       // generic-proxy writes -> visible to the tensor core's async proxy
+        // one fence for both hand-overs: the widened tile becomes visible to the tensor core's async
+        // proxy, and the reads of the packed tile (consumed by the stores above) are ordered before
+        // the TMA write that re-fills it
+        fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) mbar_arrive_cluster(op_full_leader + 8u * s);
+        if (lane == 0) { mbar_arrive(pk_empty(ps)); mbar_arrive_cluster(op_full_leader + 8u * s); }
         if (++ps == NPK) { ps = 0; pph ^= 1u; }
         if (++s == NS) { s = 0; ph ^= 1u; }
       }
@@ -299,11 +303,8 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
       const int* zws = zw_s + b * TN + half * 128;
       // all 128 accumulators of this thread's row -> registers, then the accumulator is free again
       uint32_t v[128];
-      tmem_ld_32x32(taddr, *reinterpret_cast<uint32_t(*)[32]>(v));
-      tmem_ld_32x32(taddr + 32, *reinterpret_cast<uint32_t(*)[32]>(v + 32));
-      tmem_ld_32x32(taddr + 64, *reinterpret_cast<uint32_t(*)[32]>(v + 64));
-      tmem_ld_32x32(taddr + 96, *reinterpret_cast<uint32_t(*)[32]>(v + 96));
-      tmem_wait_ld();
+      tmem_ld_32x64(taddr, v);                           // each load and its wait in one statement
+      tmem_ld_32x64(taddr + 64, v + 64);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(acc_empty_leader);

@@ -83,3 +83,31 @@ def test_gemm_persistent_many_tiles_and_status_word():
     _, acc = B.fpt_w4a4_gemm(packed_dev(qa), packed_dev(qw), dev(sw), 1.0, want_acc=True, want_y=False, ws=ws)
     assert B.fpt_check_status(ws) == B.OK
     assert np.array_equal(host(acc), int_matmul(qa, qw))
+
+
+@pytest.mark.parametrize("residual", [False, True])
+def test_gemm_many_rounds_per_cta_pair_repeatable_and_exact(residual):
+    """Several tiles per CTA pair with the slow (residual) epilogue: results must not depend on timing
+    (a register holding an in-flight tensor-memory load must never be spilled before its wait), and
+    sampled rows must match the oracle."""
+    M, N, K = 2048, 6144, 4096
+    rng = np.random.default_rng(17)
+    qa, qw = random_codes(rng, (M, K)), random_codes(rng, (N, K))
+    sw = (np.exp(rng.standard_normal(N)) * 0.01).astype(np.float32)
+    res = torch.from_numpy(rng.standard_normal((M, N)).astype(np.float32)).to(torch.bfloat16) if residual else None
+    rs = np.exp(rng.standard_normal(M)).astype(np.float32) if residual else None
+    xa, xw, xs = packed_dev(qa), packed_dev(qw), dev(sw)
+    dres, drs = (dev(res), dev(rs)) if residual else (None, None)
+    ws = B.new_workspace(B.OP_GEMM, M, N, K)
+    outs = []
+    for _ in range(4):
+        Y, _ = B.fpt_w4a4_gemm(xa, xw, xs, 0.31, residual=dres, res_scale=drs, ws=ws)
+        outs.append(Y.view(torch.int16).clone())
+    assert B.fpt_check_status(ws) == B.OK
+    for o in outs[1:]:
+        assert torch.equal(o, outs[0]), "two launches on the same inputs gave different outputs"
+    rows = np.array([0, 127, 128, 255, 256, 1023, 1024, 1791, 1792, 2047])
+    acc = int_matmul(qa[rows], qw)
+    rres = (res.float().numpy()[rows] * rs[rows, None]).astype(np.float32) if residual else None
+    ref = dequant_epilogue(acc, sw, np.float32(0.31), None, rres)
+    assert assert_bf16_close(bf16_host(outs[0].view(torch.bfloat16))[rows], ref, "Y rows") == 0
