@@ -250,6 +250,38 @@ int fpt_decoder_mlp(void* stream, const void* X, int M, int d, int d_ff,
                     const float* s_prev, float* s_out, int add_residual, int mid_hadamard,
                     void* Y, void* workspace, size_t workspace_bytes);
 
+/*
+ * The attention block of a decoder layer in the normalised-residual form of Sec. 3.1.3, as two
+ * calls around the caller's own attention (RoPE, softmax(QK^T) V; kept in 16-bit floating point
+ * in the paper's timing runs, App. J "Setup").  The sequence scaler S_n sits at the attention
+ * output ("ap" in the placement table of App. A): a per-token scale commutes with the BMMs and
+ * with the bias-free output projection (Sec. 3.1.3, after Eq. 5).
+ *
+ * fpt_decoder_attn_qkv:
+ *   X~ = RMSNorm(X),  S_n = S_{n-1} * r,  r = 1 / sqrt(mean_k X^2 + eps)    (X is Z~_{n-1}; Eq. 7)
+ *   QKV = W4A4 linear of X~ with the fused weight Wqkv_q [n_qkv, d/2]        grid qp_in
+ *         (query || key || value rows, the pre-RoPE and value transforms of Sec. 3.1.1-3.1.2
+ *         already merged into it); QKV [M, n_qkv] bf16 carries no S_n: RMSNorm removed it.
+ *   s_prev [M] or NULL (= 1); s_out [M] out: S_n;  r_out [M] out: r (scales the residual later).
+ * fpt_decoder_attn_out:
+ *   A [M, k_o] bf16: the caller's attention output (heads concatenated)
+ *   codes = grid_qp_ap(A * S_n)                                             (scaler at "ap")
+ *   Y~ = W4A4 output projection with Wo_q [d, k_o/2]  (= S_n * Y_n, Eq. 5)
+ *   Y  = bf16(Y~ + X * r)  if X != NULL   (Z~_n = X~_n + Y~_n;  X is the Z~_{n-1} given to
+ *        fpt_decoder_attn_qkv, r its r_out)                     else bf16(Y~)
+ * wsum_* [N] int32: required when the grid is asymmetric, else NULL.
+ * Shapes as fpt_w4a4_linear; workspace: fpt_workspace_bytes(FPT_OP_LINEAR, M, n_qkv, d) resp.
+ * (FPT_OP_LINEAR, M, d, k_o) bytes.  The two calls may share one workspace.
+ */
+int fpt_decoder_attn_qkv(void* stream, const void* X, int M, int d,
+                         const uint8_t* Wqkv_q, const void* sw_qkv, int scale_dtype, const int32_t* wsum_qkv,
+                         int n_qkv, const fpt_qparams* qp_in, float eps, const float* s_prev,
+                         float* s_out, float* r_out, void* QKV, void* workspace, size_t workspace_bytes);
+int fpt_decoder_attn_out(void* stream, const void* A, int M, int k_o,
+                         const uint8_t* Wo_q, const void* sw_o, int scale_dtype, const int32_t* wsum_o, int d,
+                         const fpt_qparams* qp_ap, const float* s_n, const void* X, const float* r,
+                         void* Y, void* workspace, size_t workspace_bytes);
+
 /* Bytes of caller-provided scratch an entry point needs (op = FPT_OP_*).
  * FPT_OP_LINEAR / FPT_OP_GEMM: (M, N, K); FPT_OP_MLP: (M, d_ff, d). */
 size_t fpt_workspace_bytes(int op, int M, int N, int K);

@@ -21,7 +21,8 @@ Modules and the passages they follow
                 function preservation
     hadamard    block-wise Hadamard transform at the down-projection input (Sec. 3.1 last
                 paragraph; App. A transform table; App. D "Hadamard non-powers of 2")
-    linear      the composed entry points (one W4A4 linear; one SwiGLU MLP block)
+    linear      the composed entry points (one W4A4 linear; one SwiGLU MLP block; the attention
+                block's two projections around the caller's attention)
 
 Parity status: every function is pinned by a CPU test (tests/test_oracle_*.py)
 against something other than itself, with two exceptions that cannot be pinned

@@ -11,6 +11,11 @@ decoder_mlp : one SwiGLU MLP block in the normalised-residual form of Sec. 3.1.3
                      (the scaler placed at the down-projection input)
               Y~_n = W4A4 down projection of S_n * m  (= S_n * Y_n, Eq. 5)
               Z~_n = X~_n + Y~_n   when the residual is requested
+decoder_attn_qkv / decoder_attn_out : the attention block in the same form, split around the
+              attention itself (which stays in 16-bit floating point, App. J "Setup"):
+              X~_n = RMSNorm(Z~_{n-1}),  S_n = S_{n-1} / ||Z~_{n-1}||_R,  QKV = W4A4 linear of X~_n;
+              then, with the scaler at the attention output ("ap", App. A placement table):
+              Y~_n = W4A4 output projection of S_n * A  (= S_n * Y_n, Eq. 5),  Z~_n = X~_n + Y~_n
 """
 import numpy as np
 
@@ -61,3 +66,26 @@ def decoder_mlp(x, wg_q, sw_g, wu_q, sw_u, wd_q, sw_d, qp_in, qp_mid, eps=1e-5,
         res = (np.asarray(x, dtype=F32) * r[:, None]).astype(F32)     # X~_n = Z~_{n-1} / rho
     y = dequant_epilogue(acc_d, sw_d, qp_mid.scale, None, res)
     return dict(xq=xq, g=g, u=u, m=m, mq=mq, acc_d=acc_d, y=y, s_out=s_n, r=r)
+
+
+def decoder_attn_qkv(x, wqkv_q, sw_qkv, qp_in, eps=1e-5, s_prev=None, wsum=None):
+    """Returns dict(xq, acc, qkv, s_out, r).  `wqkv_q` holds the query, key and value rows with the
+    mergeable transforms (Sec. 3.1.1, 3.1.2) already folded in; RMSNorm's output carries no
+    per-token scale, so neither does QKV."""
+    xq, s_n, p, r = act_quant(x, qp_in, rmsnorm=True, scale_input=False, eps=eps, s_in=s_prev)
+    acc = int_matmul(xq, wqkv_q, qp_in.z)
+    qkv = dequant_epilogue(acc, sw_qkv, qp_in.scale)
+    return dict(xq=xq, acc=acc, qkv=qkv, s_out=s_n, r=r)
+
+
+def decoder_attn_out(a, wo_q, sw_o, qp_ap, s_n, x=None, r=None):
+    """Returns dict(aq, acc, y).  `a` is the attention output (bf16 values); the grid sees
+    a * S_n; with `x` (the Z~_{n-1} that entered the block) and its `r`, the normalised residual
+    X~_n = x * r is added in float32 before the one rounding to bf16."""
+    aq, _, _, _ = act_quant(a, qp_ap, rmsnorm=False, scale_input=True, s_in=s_n)
+    acc = int_matmul(aq, wo_q, qp_ap.z)
+    res = None
+    if x is not None:
+        res = (np.asarray(x, dtype=F32) * np.asarray(r, dtype=F32)[:, None]).astype(F32)
+    y = dequant_epilogue(acc, sw_o, qp_ap.scale, None, res)
+    return dict(aq=aq, acc=acc, y=y)

@@ -22,7 +22,8 @@ POST_NONE, POST_INVERSE_OF_PRE, POST_VECTOR = 0, 1, 2
 OP_LINEAR, OP_MLP, OP_GEMM = 0, 1, 2
 
 EXPORTS = ["fpt_version", "fpt_strerror", "fpt_quantize_weights", "fpt_interleave_gate_up", "fpt_act_quant", "fpt_hadamard_quant",
-           "fpt_w4a4_gemm", "fpt_w4a4_linear", "fpt_w4a4_linear_static", "fpt_decoder_mlp", "fpt_workspace_bytes", "fpt_reset_status",
+           "fpt_w4a4_gemm", "fpt_w4a4_linear", "fpt_w4a4_linear_static", "fpt_decoder_mlp", "fpt_decoder_attn_qkv",
+           "fpt_decoder_attn_out", "fpt_workspace_bytes", "fpt_reset_status",
            "fpt_check_status"]
 
 
@@ -64,6 +65,8 @@ def lib():
         L.fpt_w4a4_linear_static.argtypes = [vp, vp, ci, ci, vp, vp, ci, vp, ci, qp, ci, cf, vp, ci, vp, vp, vp]
         L.fpt_decoder_mlp.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp, vp, ci, qp, qp, cf, vp, vp, ci, ci, vp, vp, sz]
         L.fpt_hadamard_quant.argtypes = [vp, vp, ci, ci, ci, qp, ci, vp, vp]
+        L.fpt_decoder_attn_qkv.argtypes = [vp, vp, ci, ci, vp, vp, ci, vp, ci, qp, cf, vp, vp, vp, vp, vp, sz]
+        L.fpt_decoder_attn_out.argtypes = [vp, vp, ci, ci, vp, vp, ci, vp, ci, qp, vp, vp, vp, vp, vp, sz]
         L.fpt_workspace_bytes.restype = sz
         L.fpt_workspace_bytes.argtypes = [ci, ci, ci, ci]
         L.fpt_reset_status.argtypes = [vp, vp]
@@ -228,3 +231,34 @@ def fpt_decoder_mlp(X, Wgu_q, sw_gu, Wd_q, sw_d, qp_in, qp_mid, eps=1e-5, s_prev
                                  ws.numel()),
            "fpt_decoder_mlp")
     return Y, s_out
+
+
+def fpt_decoder_attn_qkv(X, Wqkv_q, sw_qkv, qp_in, eps=1e-5, s_prev=None, wsum=None, ws=None, QKV=None):
+    """First half of the attention block -> (QKV bf16 [M, n_qkv], S_n f32 [M], r f32 [M])."""
+    M, d = X.shape
+    n_qkv = Wqkv_q.shape[0]
+    if ws is None:
+        ws = new_workspace(OP_LINEAR, M, n_qkv, d, X.device)
+    if QKV is None:
+        QKV = torch.empty((M, n_qkv), dtype=torch.bfloat16, device=X.device)
+    s_out = torch.empty((M,), dtype=torch.float32, device=X.device)
+    r_out = torch.empty((M,), dtype=torch.float32, device=X.device)
+    _check(lib().fpt_decoder_attn_qkv(_stream(), _ptr(X), M, d, _ptr(Wqkv_q), _ptr(sw_qkv), _scale_dtype(sw_qkv),
+                                      _ptr(wsum), n_qkv, ctypes.byref(qp_in), eps, _ptr(s_prev), _ptr(s_out),
+                                      _ptr(r_out), _ptr(QKV), _ptr(ws), ws.numel()), "fpt_decoder_attn_qkv")
+    return QKV, s_out, r_out
+
+
+def fpt_decoder_attn_out(A, Wo_q, sw_o, qp_ap, s_n, X=None, r=None, wsum=None, ws=None, Y=None):
+    """Second half of the attention block: scaler at the attention output, output projection,
+    optional normalised residual -> Y bf16 [M, d]."""
+    M, k_o = A.shape
+    d = Wo_q.shape[0]
+    if ws is None:
+        ws = new_workspace(OP_LINEAR, M, d, k_o, A.device)
+    if Y is None:
+        Y = torch.empty((M, d), dtype=torch.bfloat16, device=A.device)
+    _check(lib().fpt_decoder_attn_out(_stream(), _ptr(A), M, k_o, _ptr(Wo_q), _ptr(sw_o), _scale_dtype(sw_o), _ptr(wsum),
+                                      d, ctypes.byref(qp_ap), _ptr(s_n), _ptr(X), _ptr(r), _ptr(Y), _ptr(ws),
+                                      ws.numel()), "fpt_decoder_attn_out")
+    return Y

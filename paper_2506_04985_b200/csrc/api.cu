@@ -204,3 +204,49 @@ extern "C" int fpt_decoder_mlp(void* stream, const void* X, int M, int d, int d_
   return fpt_w4a4_gemm(stream, Mq, Wd_q, M, d, d_ff, sw_d, scale_dtype, nullptr, qp_mid->scale, 1, 0, nullptr,
                        add_residual ? X : nullptr, add_residual ? r_ws : nullptr, Y, nullptr, workspace, gemm_ws);
 }
+
+extern "C" int fpt_decoder_attn_qkv(void* stream, const void* X, int M, int d, const uint8_t* Wqkv_q, const void* sw_qkv,
+                                    int scale_dtype, const int32_t* wsum_qkv, int n_qkv, const fpt_qparams* qp_in,
+                                    float eps, const float* s_prev, float* s_out, float* r_out, void* QKV,
+                                    void* workspace, size_t workspace_bytes) {
+  if (!X || !Wqkv_q || !sw_qkv || !QKV || !s_out || !r_out) return FPT_ERR_BAD_ARG;
+  int rc = check_qp(qp_in);
+  if (rc) return rc;
+  rc = check_gemm_shape(M, n_qkv, d);
+  if (rc) return rc;
+  if (!qp_in->symmetric && !wsum_qkv) return FPT_ERR_BAD_ARG;
+  if (((uintptr_t)X | (uintptr_t)Wqkv_q | (uintptr_t)QKV | (uintptr_t)workspace) & 15) return FPT_ERR_ALIGNMENT;
+  if (!workspace || workspace_bytes < fpt_workspace_bytes(FPT_OP_LINEAR, M, n_qkv, d)) return FPT_ERR_WORKSPACE;
+  const size_t gemm_ws = kStatusBytes + gemm_scratch_bytes(M);
+  uint8_t* Xq = reinterpret_cast<uint8_t*>(workspace) + gemm_ws;
+  // X~ = RMSNorm(X) on the grid qp_in; S_n = S_{n-1} * r; r kept for the residual
+  if (act_quant_launch((cudaStream_t)stream, X, M, d, d, qp_in, FPT_RMSNORM, eps, nullptr, s_prev, Xq, s_out, nullptr,
+                       r_out) != cudaSuccess)
+    return FPT_ERR_CUDA;
+  return fpt_w4a4_gemm(stream, Xq, Wqkv_q, M, n_qkv, d, sw_qkv, scale_dtype, wsum_qkv, qp_in->scale, qp_in->symmetric,
+                       qp_in->zero_point, nullptr, nullptr, nullptr, QKV, nullptr, workspace, gemm_ws);
+}
+
+extern "C" int fpt_decoder_attn_out(void* stream, const void* A, int M, int k_o, const uint8_t* Wo_q, const void* sw_o,
+                                    int scale_dtype, const int32_t* wsum_o, int d, const fpt_qparams* qp_ap,
+                                    const float* s_n, const void* X, const float* r, void* Y, void* workspace,
+                                    size_t workspace_bytes) {
+  if (!A || !Wo_q || !sw_o || !Y || !s_n) return FPT_ERR_BAD_ARG;
+  if (X && !r) return FPT_ERR_BAD_ARG;
+  int rc = check_qp(qp_ap);
+  if (rc) return rc;
+  rc = check_gemm_shape(M, d, k_o);
+  if (rc) return rc;
+  if (!qp_ap->symmetric && !wsum_o) return FPT_ERR_BAD_ARG;
+  if (((uintptr_t)A | (uintptr_t)Wo_q | (uintptr_t)Y | (uintptr_t)X | (uintptr_t)workspace) & 15) return FPT_ERR_ALIGNMENT;
+  if (!workspace || workspace_bytes < fpt_workspace_bytes(FPT_OP_LINEAR, M, d, k_o)) return FPT_ERR_WORKSPACE;
+  const size_t gemm_ws = kStatusBytes + gemm_scratch_bytes(M);
+  uint8_t* Aq = reinterpret_cast<uint8_t*>(workspace) + gemm_ws;
+  // the sequence scaler at the attention output: the grid sees A * S_n
+  if (act_quant_launch((cudaStream_t)stream, A, M, k_o, k_o, qp_ap, FPT_SCALE_INPUT, 0.0f, nullptr, s_n, Aq, nullptr,
+                       nullptr, nullptr) != cudaSuccess)
+    return FPT_ERR_CUDA;
+  // output projection; the normalised residual X * r joins before the final rounding
+  return fpt_w4a4_gemm(stream, Aq, Wo_q, M, d, k_o, sw_o, scale_dtype, wsum_o, qp_ap->scale, qp_ap->symmetric,
+                       qp_ap->zero_point, nullptr, X, X ? r : nullptr, Y, nullptr, workspace, gemm_ws);
+}

@@ -137,3 +137,50 @@ def test_config2_attention_projections_sampled():
     ref = OL.w4a4_linear(aof[rows], cw, d, oqp(qp_o), False, True, 1e-5, s_in.numpy()[rows])
     assert len(np.unique(ref["codes"])) >= 8
     assert assert_bf16_close(bf16_host(Y)[rows], ref["y"], "cfg2 o") == 0
+
+
+@pytest.mark.parametrize("M,d,n_q,n_kv,with_prev,residual,symmetric",
+                         [(96, 256, 256, 64, True, True, True), (300, 1024, 1024, 256, True, True, True),
+                          (33, 512, 512, 128, False, False, True), (513, 256, 256, 128, True, True, False)])
+def test_decoder_attention_projections_parity(M, d, n_q, n_kv, with_prev, residual, symmetric):
+    """fpt_decoder_attn_qkv -> (an attention stand-in on the host) -> fpt_decoder_attn_out against the
+    oracle's two halves on the same values: codes-derived outputs, S_n and r bit-exact."""
+    seed = 5
+    x = synth.activations(M, d, seed, "attn/x", law="student_t3", outlier_frac=0.005, outlier_gain=50.0)
+    wqkv = synth.weights(n_q + 2 * n_kv, d, 0.02, seed, "attn/wqkv")
+    wo = synth.weights(d, n_q, 0.02, seed, "attn/wo")
+    s_prev = synth.per_token_scale(M, seed, "attn/s") if with_prev else None
+    xf = synth.f32(x)
+    cqkv, sqkv, wsum_qkv = OQ.quantize_weights(synth.f32(wqkv))
+    co, so, wsum_o = OQ.quantize_weights(synth.f32(wo))
+    r = OQ.rms_reciprocal(xf, 1e-5)
+    if symmetric:
+        qp_in = B.QParams(4, True, float(OQ.calibrate_static_scale(xf[:64] * r[:64, None], OQ.QParams())), 0)
+    else:
+        qp_in = B.QParams(4, False, 0.3, 7)
+    wq_d, sw_d, ws_d = B.fpt_quantize_weights(dev(wqkv), want_wsum=not symmetric)
+    wo_d, swo_d, wso_d = B.fpt_quantize_weights(dev(wo), want_wsum=not symmetric)
+    xd = dev(x)
+    QKV, s_n, r_out = B.fpt_decoder_attn_qkv(xd, wq_d, sw_d, qp_in, 1e-5, None if s_prev is None else dev(s_prev),
+                                             wsum=ws_d)
+    ref1 = OL.decoder_attn_qkv(xf, cqkv, sqkv, oqp(qp_in), 1e-5, None if s_prev is None else s_prev.numpy())
+    assert np.array_equal(host(s_n), ref1["s_out"]) and np.array_equal(host(r_out), ref1["r"])
+    assert len(np.unique(ref1["xq"])) >= 8
+    assert assert_bf16_close(bf16_host(QKV), ref1["qkv"], "attn QKV") == 0
+    # stand-in for the caller's attention: any bf16 [M, n_q] tensor computed from QKV will do for parity;
+    # a causal running mean of the value heads keeps it data-dependent
+    qkv = bf16_host(QKV)
+    v = qkv[:, n_q + n_kv:]
+    run = np.cumsum(v.astype(np.float64), axis=0) / np.arange(1, M + 1)[:, None]
+    a = synth.to_bf16(np.tile(run, (1, n_q // n_kv)) + 0.25 * qkv[:, :n_q])
+    af = synth.f32(a)
+    if symmetric:
+        qp_ap = B.QParams(4, True, float(OQ.calibrate_static_scale(af[:64] * ref1["s_out"][:64, None], OQ.QParams())), 0)
+    else:
+        qp_ap = B.QParams(4, False, float(np.abs(af * ref1["s_out"][:, None]).max() / 7.5), 8)
+    Y = B.fpt_decoder_attn_out(dev(a), wo_d, swo_d, qp_ap, s_n, xd if residual else None, r_out if residual else None,
+                               wsum=wso_d)
+    ref2 = OL.decoder_attn_out(af, co, so, oqp(qp_ap), ref1["s_out"], xf if residual else None,
+                               ref1["r"] if residual else None)
+    assert len(np.unique(ref2["aq"])) >= 6
+    assert assert_bf16_close(bf16_host(Y), ref2["y"], "attn Y") == 0

@@ -7,6 +7,7 @@ from oracle.quantizers import QParams
 from oracle.int_matmul import int_matmul, int_matmul_bruteforce
 from oracle.epilogue import dequant_epilogue, inverse_of_pre
 from oracle import linear as L
+from oracle import transforms as T
 
 F32 = np.float32
 
@@ -128,3 +129,75 @@ def test_decoder_mlp_tracks_float64_block_and_scale_bookkeeping():
     assert np.linalg.norm(out_nr["y"] - y_ref) / np.linalg.norm(y_ref) < 0.45
     # exact integer accumulators whichever way they are computed
     assert np.array_equal(out["acc_d"][:2, :3].astype(np.int64), int_matmul_bruteforce(out["mq"][:2], cd[:3]))
+
+
+def _attention_core_f64(q, k, v, d_head, m, thetas):
+    """softmax(rope(q) rope(k)^T / sqrt(d)) v per head, causal, grouped-query; float64."""
+    Lq = q.shape[0]
+    pos = np.arange(Lq)
+    mask = np.triu(np.ones((Lq, Lq), dtype=bool), k=1)
+    heads = []
+    for j in range(q.shape[1] // d_head):
+        h = j // m
+        qj = T.apply_rope(q[:, j * d_head:(j + 1) * d_head], pos, thetas, "half")
+        kh = T.apply_rope(k[:, h * d_head:(h + 1) * d_head], pos, thetas, "half")
+        lg = np.where(mask, -np.inf, qj @ kh.T / np.sqrt(d_head))
+        a = np.exp(lg - lg.max(axis=-1, keepdims=True))
+        heads.append((a / a.sum(axis=-1, keepdims=True)) @ v[:, h * d_head:(h + 1) * d_head])
+    return np.concatenate(heads, axis=1)
+
+
+def test_decoder_attention_projections_track_float64_block_and_scale_bookkeeping():
+    """The two halves of the attention block around a float64 attention core: S_n bookkeeping exact
+    (Eq. 7), Z~_n = X~_n + S_n * Y_n (Eq. 5) within what two 4-bit grids allow, the scaler at the
+    attention output commutes with the output projection, integer accumulators by brute force."""
+    rng = np.random.default_rng(21)
+    M, d, d_head, n_kv, m = 40, 256, 32, 2, 4
+    n_q = n_kv * m
+    x = bf16.round_to_bf16(rng.standard_normal((M, d)).astype(F32) * np.exp(rng.standard_normal((M, 1))).astype(F32))
+    s_prev = np.exp(rng.standard_normal(M) * 0.5).astype(F32)
+    wq, wk, wv = (bf16.round_to_bf16((rng.standard_normal((n, d)) * 0.06).astype(F32))
+                  for n in (n_q * d_head, n_kv * d_head, n_kv * d_head))
+    wo = bf16.round_to_bf16((rng.standard_normal((d, n_q * d_head)) * 0.06).astype(F32))
+    wqkv = np.concatenate([wq, wk, wv], axis=0)
+    cqkv, sqkv, _ = Q.quantize_weights(wqkv)
+    co, so, _ = Q.quantize_weights(wo)
+    r = Q.rms_reciprocal(x, 1e-5)
+    xn = (x * r[:, None]).astype(np.float64)
+    qp_in = QParams(4, True, float(Q.calibrate_static_scale(xn, QParams())))
+    first = L.decoder_attn_qkv(x, cqkv, sqkv, qp_in, 1e-5, s_prev)
+    assert np.array_equal(first["s_out"], (r * s_prev).astype(F32))          # Eq. 7
+    assert np.array_equal(first["r"], r)
+    qkv_ref = xn @ wqkv.astype(np.float64).T
+    assert np.linalg.norm(first["qkv"] - qkv_ref) / np.linalg.norm(qkv_ref) < 0.25
+    assert np.array_equal(first["acc"][:2, :3].astype(np.int64), int_matmul_bruteforce(first["xq"][:2], cqkv[:3]))
+    # QKV carries no per-token scale: another S_{n-1} changes S_n only
+    again = L.decoder_attn_qkv(x, cqkv, sqkv, qp_in, 1e-5, None)
+    assert np.array_equal(again["qkv"], first["qkv"]) and np.array_equal(again["s_out"], r)
+    # the caller's attention (float64 here) on the reference projections
+    thetas = 10000.0 ** (-np.arange(d_head // 2) / (d_head // 2))
+    nq, nk = n_q * d_head, n_kv * d_head
+    a_ref = _attention_core_f64(qkv_ref[:, :nq], qkv_ref[:, nq:nq + nk], qkv_ref[:, nq + nk:], d_head, m, thetas)
+    a = bf16.round_to_bf16(a_ref.astype(F32))
+    s_n = first["s_out"]
+    qp_ap = QParams(4, True, float(Q.calibrate_static_scale(a_ref * s_n[:, None].astype(np.float64), QParams())))
+    second = L.decoder_attn_out(a, co, so, qp_ap, s_n, x, r)
+    y_ref = (a_ref * s_n[:, None].astype(np.float64)) @ wo.astype(np.float64).T     # S_n * Y_n  (Eq. 5)
+    z_ref = xn + y_ref                                                               # Z~_n = X~_n + Y~_n
+    err = np.linalg.norm(second["y"] - z_ref) / np.linalg.norm(z_ref)
+    assert err < 0.35
+    # ... and nowhere near the block with the scaler left out, or the residual left unnormalised
+    assert np.linalg.norm(second["y"] - (xn + a_ref @ wo.astype(np.float64).T)) / np.linalg.norm(z_ref) > 2 * err
+    assert np.linalg.norm(second["y"] - (x.astype(np.float64) + y_ref)) / np.linalg.norm(z_ref) > 2 * err
+    no_res = L.decoder_attn_out(a, co, so, qp_ap, s_n)
+    assert np.linalg.norm(no_res["y"] - y_ref) / np.linalg.norm(y_ref) < 0.45
+    assert np.array_equal(second["acc"], no_res["acc"])
+    assert np.array_equal(second["acc"][:2, :3].astype(np.int64), int_matmul_bruteforce(second["aq"][:2], co[:3]))
+    # the scaler commutes with the projection: powers of two move through the grid exactly
+    two = np.full(M, 4.0, dtype=F32)
+    scaled = L.decoder_attn_out(a, co, so, QParams(4, True, qp_ap.scale * 4.0), s_n * two)
+    assert np.array_equal(scaled["aq"], second["aq"])
+    assert np.array_equal(scaled["y"], (no_res["y"] * 4.0).astype(F32))
+    # and it matters where the scale is: without S_n the same grid clips differently
+    unscaled = L.decoder_attn_out(a, co, so, qp_ap, np.ones(M, dtype=F32))
+    assert not np.array_equal(unscaled["aq"], second["aq"])
