@@ -19,7 +19,7 @@ decoder_attn_qkv / decoder_attn_out : the attention block in the same form, spli
 """
 import numpy as np
 
-from .quantizers import QParams, act_quant, silu_mul_quant
+from .quantizers import QParams, act_quant, act_quant_dynamic, silu_mul_quant
 from .int_matmul import int_matmul
 from .epilogue import dequant_epilogue, inverse_of_pre
 from .hadamard import block_hadamard_f32
@@ -89,3 +89,21 @@ def decoder_attn_out(a, wo_q, sw_o, qp_ap, s_n, x=None, r=None):
         res = (np.asarray(x, dtype=F32) * np.asarray(r, dtype=F32)[:, None]).astype(F32)
     y = dequant_epilogue(acc, sw_o, qp_ap.scale, None, res)
     return dict(aq=aq, acc=acc, y=y)
+
+
+def w4a4_linear_dynamic(x, wq, sw, bits=4, rmsnorm=True, scale_input=False, eps=1e-5, s_in=None,
+                        post_mode=POST_NONE, post=None):
+    """The linear with the dynamic activation quantiser (App. B "Dynamic quantization"; the second
+    timing table of App. J): per-token grid D_t, integer matmul, and the scale factors
+    y = bf16(((float)acc * sw[n]) * c_t) with c_t = D_t, D_t * (1/p_t) or D_t * post[t].
+    Returns dict(codes, delta, acc, y, s_out, p, r)."""
+    codes, delta, s_out, p, r = act_quant_dynamic(x, bits, rmsnorm, scale_input, eps, s_in)
+    acc = int_matmul(codes, wq, 0)
+    if post_mode == POST_NONE:
+        c = delta
+    elif post_mode == POST_INVERSE_OF_PRE:
+        c = (delta * inverse_of_pre(p)).astype(F32)
+    else:
+        c = (delta * np.asarray(post, dtype=F32)).astype(F32)
+    y = dequant_epilogue(acc, sw, 1.0, c)
+    return dict(codes=codes, delta=delta, acc=acc, y=y, s_out=s_out, p=p, r=r)

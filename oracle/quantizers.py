@@ -22,6 +22,8 @@ the same readings in its header, in its own words)
     x^ = D*q; asymmetric q = clamp(rne(x/D) + z, 0, 2^b - 1), x^ = D*(q - z);
   * rounding is to nearest with ties to even;
   * the static activation scale is one scalar per tensor;
+  * the dynamic variant (App. B) uses, per token, the symmetric grid that ends at the
+    token's largest magnitude;
   * arithmetic precision: float32 with one rounding per operation and no fused
     multiply-add, except the sum of squares of the RMS, which is accumulated in
     float64 and rounded once;
@@ -193,6 +195,37 @@ def act_quant(x, qp, rmsnorm=True, scale_input=False, eps=1e-5, s_in=None):
     u = (x * p[:, None]) * inv_d                                   # two roundings, no FMA
     codes = round_clamp(u, qp.z, qp.qmin, qp.qmax)
     return codes, s_out, p, r
+
+
+def act_quant_dynamic(x, bits=4, rmsnorm=True, scale_input=False, eps=1e-5, s_in=None):
+    """Dynamic activation quantiser: one grid per token, computed at run time (App. B, "Dynamic
+    quantization": the extreme activation values are reduced over the last dimension for each
+    token and the resulting scale factor is applied to each value).
+
+    Reading taken (the paper gives no formula): the symmetric grid whose end is the token's
+    largest magnitude,
+      v_tk    = x_tk * p_t                          p_t as in act_quant
+      m_t     = max_k |v_tk|
+      D_t     = m_t / qmax   (float32 division);  D_t = 1 when m_t is zero, infinite or NaN
+      q_tk    = clamp(rne(v_tk * (1 / D_t)), qmin, qmax)      (1 / D_t: float32 division)
+    Returns (codes, D [M] float32, S_out, p, r).
+    """
+    x = np.asarray(x, dtype=F32)
+    M = x.shape[0]
+    qp = QParams(bits, True, 1.0, 0)
+    r = rms_reciprocal(x, eps) if rmsnorm else np.ones(M, dtype=F32)
+    s = None if s_in is None else np.asarray(s_in, dtype=F32)
+    p = (r * s).astype(F32) if (scale_input and s is not None) else r
+    s_out = (r * s).astype(F32) if s is not None else r
+    v = (x * p[:, None]).astype(F32)
+    with np.errstate(invalid="ignore"):
+        m = np.max(np.abs(v), axis=1).astype(F32)              # NaN propagates
+        ok = np.isfinite(m) & (m > 0)
+        delta = np.where(ok, m / F32(qp.qmax), F32(1.0)).astype(F32)
+    inv = (F32(1.0) / delta).astype(F32)
+    u = (v * inv[:, None]).astype(F32)
+    codes = round_clamp(u, 0, qp.qmin, qp.qmax)
+    return codes, delta, s_out, p, r
 
 
 # --------------------------------------------------------------------------- #

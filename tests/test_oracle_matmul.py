@@ -201,3 +201,50 @@ def test_decoder_attention_projections_track_float64_block_and_scale_bookkeeping
     # and it matters where the scale is: without S_n the same grid clips differently
     unscaled = L.decoder_attn_out(a, co, so, qp_ap, np.ones(M, dtype=F32))
     assert not np.array_equal(unscaled["aq"], second["aq"])
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_dynamic_linear_on_grid_inputs_reduce_to_a_float64_matmul(bits):
+    """Rows that lie on their own dynamic grid (x = c_t * q, |q| reaching qmax, c_t a power of two)
+    are quantised without error, so the whole dynamic linear equals the float64 product."""
+    rng = np.random.default_rng(33)
+    M, K, N = 24, 256, 40
+    qmax = 2 ** (bits - 1) - 1
+    qa = rng.integers(-qmax, qmax + 1, (M, K))
+    qa[np.arange(M), rng.integers(0, K, M)] = qmax * rng.choice([-1, 1], M)
+    c = np.exp2(rng.integers(-6, 3, M))
+    x = (qa * c[:, None]).astype(F32)
+    qw = rng.integers(-8, 8, (N, K)).astype(np.int8)
+    sw = np.exp2(rng.integers(-8, -3, N)).astype(F32)
+    out = L.w4a4_linear_dynamic(x, qw, sw, bits, rmsnorm=False)
+    assert np.array_equal(out["codes"], qa) and np.array_equal(out["delta"], c.astype(F32))
+    ref = x.astype(np.float64) @ (qw * sw[:, None].astype(np.float64)).T
+    assert np.array_equal(out["y"], bf16.round_to_bf16(ref.astype(F32)))
+    assert np.array_equal(out["acc"][:2, :3].astype(np.int64), int_matmul_bruteforce(qa[:2], qw[:3]))
+
+
+def test_dynamic_linear_post_modes_and_gain_over_static_on_outlier_tokens():
+    rng = np.random.default_rng(34)
+    M, K, N = 64, 512, 48
+    x = bf16.round_to_bf16((rng.standard_normal((M, K)) * np.exp(rng.standard_normal((M, 1)) * 1.5)).astype(F32))
+    w = bf16.round_to_bf16((rng.standard_normal((N, K)) * 0.05).astype(F32))
+    cw, sw, _ = Q.quantize_weights(w)
+    ref = x.astype(np.float64) @ w.astype(np.float64).T
+    dyn = L.w4a4_linear_dynamic(x, cw, sw, 4, rmsnorm=False)
+    e_dyn = np.linalg.norm(dyn["y"] - ref) / np.linalg.norm(ref)
+    d_static = float(Q.calibrate_static_scale(x.astype(np.float64), QParams()))
+    sta = L.w4a4_linear(x, cw, sw, QParams(4, True, d_static), rmsnorm=False)
+    e_sta = np.linalg.norm(sta["y"] - ref) / np.linalg.norm(ref)
+    assert e_dyn < 0.3 and e_dyn < 0.7 * e_sta             # per-token grids absorb the norm disparity (App. B)
+    y8 = L.w4a4_linear_dynamic(x, cw, sw, 8, rmsnorm=False)["y"]
+    assert np.linalg.norm(y8 - ref) / np.linalg.norm(ref) < e_dyn
+    ref_wq = x.astype(np.float64) @ (cw.astype(np.float64) * sw[:, None].astype(np.float64)).T
+    assert np.linalg.norm(y8 - ref_wq) / np.linalg.norm(ref_wq) < 0.02    # 8-bit activations: only the weight grid's error remains
+    # post modes: with the RMSNorm in front, INVERSE_OF_PRE undoes the normalisation, VECTOR applies any vector
+    r = Q.rms_reciprocal(x, 1e-5)
+    inv = L.w4a4_linear_dynamic(x, cw, sw, 4, rmsnorm=True, post_mode=L.POST_INVERSE_OF_PRE)
+    assert np.linalg.norm(inv["y"] - ref) / np.linalg.norm(ref) < 0.3
+    vec = L.w4a4_linear_dynamic(x, cw, sw, 4, rmsnorm=True, post_mode=L.POST_VECTOR, post=np.full(M, 2.0, dtype=F32))
+    non = L.w4a4_linear_dynamic(x, cw, sw, 4, rmsnorm=True)
+    assert np.array_equal(vec["y"], (non["y"] * F32(2.0)).astype(F32))
+    assert np.array_equal(non["codes"], inv["codes"]) and np.array_equal(non["s_out"], r)

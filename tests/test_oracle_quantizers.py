@@ -276,3 +276,65 @@ def test_calibration_recovers_an_exact_grid_and_clips_tails():
         errs.append((e, di))
     best = min(errs, key=lambda p: (p[0], -p[1]))[1]
     assert float(Q.calibrate_static_scale(small, qp)) == pytest.approx(best, rel=1e-6)
+
+
+# --------------------------------------------------------------------------- #
+# dynamic (per-token) quantiser, 4 and 8 bits
+# --------------------------------------------------------------------------- #
+@pytest.mark.parametrize("bits", [4, 8])
+def test_dynamic_quantiser_grid_ends_at_the_token_maximum(bits):
+    rng = np.random.default_rng(31)
+    M, K = 64, 256
+    x = bf16.round_to_bf16((rng.standard_normal((M, K)) * np.exp(rng.standard_normal((M, 1)) * 2)).astype(F32))
+    s_in = np.exp(rng.standard_normal(M)).astype(F32)
+    qmax = 2 ** (bits - 1) - 1
+    for rmsnorm, scale_input in ((True, False), (False, True), (True, True), (False, False)):
+        codes, delta, s_out, p, r = Q.act_quant_dynamic(x, bits, rmsnorm, scale_input, 1e-5, s_in)
+        # the scale is the token's largest magnitude over qmax (float64 restatement, float32 tolerance)
+        m64 = np.max(np.abs(x.astype(np.float64)), axis=1) * p.astype(np.float64)
+        assert np.allclose(delta, m64 / qmax, rtol=3e-7)
+        # so the largest element sits on the last code, nothing is clipped, and the error is half a step
+        assert np.array_equal(np.max(np.abs(codes.astype(np.int32)), axis=1), np.full(M, qmax))
+        v = x.astype(np.float64) * p.astype(np.float64)[:, None]
+        err = np.abs(v - delta.astype(np.float64)[:, None] * codes)
+        assert np.all(err <= 0.5 * delta.astype(np.float64)[:, None] * (1 + 1e-5))
+        # per row it is the static quantiser with that row's scale
+        for t in (0, 17, M - 1):
+            ref, _, _, _ = Q.act_quant(x[t:t + 1], QParams(bits, True, float(delta[t])), rmsnorm, scale_input, 1e-5,
+                                       s_in[t:t + 1])
+            assert np.array_equal(ref[0], codes[t])
+        # bookkeeping identical to the static quantiser
+        _, s_ref, p_ref, r_ref = Q.act_quant(x, QParams(4, True, 1.0), rmsnorm, scale_input, 1e-5, s_in)
+        assert np.array_equal(s_out, s_ref) and np.array_equal(p, p_ref) and np.array_equal(r, r_ref)
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_dynamic_quantiser_equivariance_and_degenerate_rows(bits):
+    rng = np.random.default_rng(32)
+    x = bf16.round_to_bf16(rng.standard_normal((8, 128)).astype(F32))
+    c0, d0, _, _, _ = Q.act_quant_dynamic(x, bits, rmsnorm=False)
+    c1, d1, _, _, _ = Q.act_quant_dynamic(x * F32(8.0), bits, rmsnorm=False)
+    assert np.array_equal(c0, c1) and np.array_equal(d1, d0 * F32(8.0))      # powers of two move into the scale
+    c2, d2, _, _, _ = Q.act_quant_dynamic(-x, bits, rmsnorm=False)
+    assert np.array_equal(d2, d0)                                            # the grid depends on magnitudes only
+    qmax = 2 ** (bits - 1) - 1
+    assert np.array_equal(np.clip(-c0.astype(np.int32), -qmax - 1, qmax), c2.astype(np.int32))
+    # with the RMSNorm in front, a per-token factor on the input changes nothing at all (eps = 0)
+    f = np.exp2(rng.integers(-3, 4, 8)).astype(F32)
+    c3, d3, _, _, _ = Q.act_quant_dynamic(x, bits, rmsnorm=True, eps=0.0)
+    c4, d4, _, _, _ = Q.act_quant_dynamic(x * f[:, None], bits, rmsnorm=True, eps=0.0)
+    assert np.array_equal(c3, c4) and np.array_equal(d3, d4)
+    # an outlier token gets a wider grid than its neighbours, the others keep theirs
+    y = x.copy()
+    y[3, 5] = F32(1000.0)
+    c5, d5, _, _, _ = Q.act_quant_dynamic(y, bits, rmsnorm=False)
+    assert d5[3] == F32(1000.0) / F32(qmax) and np.array_equal(np.delete(d5, 3), np.delete(d0, 3))
+    assert np.array_equal(np.delete(c5, 3, axis=0), np.delete(c0, 3, axis=0))
+    # degenerate rows: all zero -> scale 1, codes 0; Inf or NaN in the row -> scale 1, saturated / lowest code
+    z = np.zeros((3, 128), dtype=F32)
+    z[1, 0], z[1, 1], z[1, 2] = np.inf, -np.inf, 3.0
+    z[2, 0], z[2, 1] = np.nan, -2.0
+    c6, d6, _, _, _ = Q.act_quant_dynamic(z, bits, rmsnorm=False)
+    assert np.array_equal(d6, np.ones(3, dtype=F32)) and not c6[0].any()
+    assert c6[1, 0] == qmax and c6[1, 1] == -qmax - 1 and c6[1, 2] == 3
+    assert c6[2, 0] == -qmax - 1 and c6[2, 1] == -2
