@@ -147,6 +147,22 @@ int fpt_act_quant(void* stream, const void* X, int M, int K, int ldx,
                   const void* X2, const float* s_in, uint8_t* Xq, float* s_out);
 
 /*
+ * Step (1) with a DYNAMIC grid (App. B "Dynamic quantization": for each token the extreme
+ * activation values are reduced over the last dimension and the resulting scale factor is applied
+ * to every value).  The paper prints no formula; this library's reading is the symmetric grid that
+ * ends at the token's largest magnitude.  Per token t, with r_t, p_t, s_out as in fpt_act_quant:
+ *   m_t  = max_k |x_tk * p_t|
+ *   D_t  = m_t / qmax            (float32 division; qmax = 7 or 127)
+ *          D_t = 1 when m_t is zero, infinite or NaN
+ *   q_tk = clamp(rne((x_tk * p_t) * (1 / D_t)), -qmax - 1, qmax)      (1 / D_t: float32 division)
+ *   bits = 4: Xq [M, K/2] packed codes;  bits = 8: Xq [M, K] int8 codes
+ *   delta_out [M] f32 out: D_t (required);  s_in, s_out as in fpt_act_quant.
+ * flags: FPT_RMSNORM, FPT_SCALE_INPUT.
+ */
+int fpt_act_quant_dynamic(void* stream, const void* X, int M, int K, int ldx, int bits, int flags, float eps,
+                          const float* s_in, void* Xq, float* s_out, float* delta_out);
+
+/*
  * Online block-wise Hadamard transform + per-token scale + static quantise + pack, for the input of
  * the down projection (Sec. 3.1, last paragraph; App. A transform table: H_n = n^(-1/2) (x) [[1,1],[1,-1]];
  * App. D "Hadamard non-powers of 2").  The K channels are split into K / B groups of
@@ -198,6 +214,20 @@ int fpt_w4a4_linear(void* stream, const void* X, int M, int K,
                     const fpt_qparams* act_qp, int flags, float eps, const float* s_in,
                     int post_mode, const float* post,
                     void* Y, float* s_out, void* workspace, size_t workspace_bytes);
+
+/*
+ * The same linear with the dynamic activation grid of fpt_act_quant_dynamic (the paper's second
+ * timing table, App. J "Dynamic INT4 runtime"):
+ *   codes, D_t as in fpt_act_quant_dynamic;  acc as in fpt_w4a4_gemm (symmetric codes);
+ *   y[t,n] = bf16( ((float)acc * sw[n]) * c_t ),
+ *   c_t = D_t (FPT_POST_NONE), D_t * (1 / p_t) (FPT_POST_INVERSE_OF_PRE), D_t * post[t] (FPT_POST_VECTOR).
+ *   bits = 4 in this version.  workspace: fpt_workspace_bytes(FPT_OP_LINEAR, M, N, K) bytes.
+ */
+int fpt_w4a4_linear_dynamic(void* stream, const void* X, int M, int K,
+                            const uint8_t* Wq, const void* sw, int scale_dtype, int N,
+                            int bits, int flags, float eps, const float* s_in,
+                            int post_mode, const float* post,
+                            void* Y, float* s_out, void* workspace, size_t workspace_bytes);
 
 /*
  * fpt_w4a4_linear without a caller workspace.  (The paper has no counterpart: this is a

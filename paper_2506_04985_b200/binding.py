@@ -23,7 +23,8 @@ OP_LINEAR, OP_MLP, OP_GEMM = 0, 1, 2
 
 EXPORTS = ["fpt_version", "fpt_strerror", "fpt_quantize_weights", "fpt_interleave_gate_up", "fpt_act_quant", "fpt_hadamard_quant",
            "fpt_w4a4_gemm", "fpt_w4a4_linear", "fpt_w4a4_linear_static", "fpt_decoder_mlp", "fpt_decoder_attn_qkv",
-           "fpt_decoder_attn_out", "fpt_workspace_bytes", "fpt_reset_status",
+           "fpt_decoder_attn_out", "fpt_act_quant_dynamic", "fpt_w4a4_linear_dynamic", "fpt_workspace_bytes",
+           "fpt_reset_status",
            "fpt_check_status"]
 
 
@@ -65,6 +66,8 @@ def lib():
         L.fpt_w4a4_linear_static.argtypes = [vp, vp, ci, ci, vp, vp, ci, vp, ci, qp, ci, cf, vp, ci, vp, vp, vp]
         L.fpt_decoder_mlp.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp, vp, ci, qp, qp, cf, vp, vp, ci, ci, vp, vp, sz]
         L.fpt_hadamard_quant.argtypes = [vp, vp, ci, ci, ci, qp, ci, vp, vp]
+        L.fpt_act_quant_dynamic.argtypes = [vp, vp, ci, ci, ci, ci, ci, cf, vp, vp, vp, vp]
+        L.fpt_w4a4_linear_dynamic.argtypes = [vp, vp, ci, ci, vp, vp, ci, ci, ci, ci, cf, vp, ci, vp, vp, vp, vp, sz]
         L.fpt_decoder_attn_qkv.argtypes = [vp, vp, ci, ci, vp, vp, ci, vp, ci, qp, cf, vp, vp, vp, vp, vp, sz]
         L.fpt_decoder_attn_out.argtypes = [vp, vp, ci, ci, vp, vp, ci, vp, ci, qp, vp, vp, vp, vp, vp, sz]
         L.fpt_workspace_bytes.restype = sz
@@ -262,3 +265,32 @@ def fpt_decoder_attn_out(A, Wo_q, sw_o, qp_ap, s_n, X=None, r=None, wsum=None, w
                                       d, ctypes.byref(qp_ap), _ptr(s_n), _ptr(X), _ptr(r), _ptr(Y), _ptr(ws),
                                       ws.numel()), "fpt_decoder_attn_out")
     return Y
+
+
+def fpt_act_quant_dynamic(X, bits=4, flags=RMSNORM, eps=1e-5, s_in=None, want_s_out=True, out=None):
+    """Dynamic per-token grid -> (codes uint8 [M, K/2] or int8 [M, K], s_out f32 [M] or None, delta f32 [M])."""
+    M, K = X.shape
+    if out is None:
+        out = (torch.empty((M, K // 2), dtype=torch.uint8, device=X.device) if bits == 4
+               else torch.empty((M, K), dtype=torch.int8, device=X.device))
+    s_out = torch.empty((M,), dtype=torch.float32, device=X.device) if want_s_out else None
+    delta = torch.empty((M,), dtype=torch.float32, device=X.device)
+    _check(lib().fpt_act_quant_dynamic(_stream(), _ptr(X), M, K, X.stride(0), bits, flags, eps, _ptr(s_in), _ptr(out),
+                                       _ptr(s_out), _ptr(delta)), "fpt_act_quant_dynamic")
+    return out, s_out, delta
+
+
+def fpt_w4a4_linear_dynamic(X, Wq, sw, bits=4, flags=RMSNORM, eps=1e-5, s_in=None, post_mode=POST_NONE, post=None,
+                            want_s_out=True, ws=None, Y=None):
+    """One linear with the dynamic activation grid -> (Y bf16 [M, N], s_out f32 [M] or None)."""
+    M, K = X.shape
+    N = Wq.shape[0]
+    if ws is None:
+        ws = new_workspace(OP_LINEAR, M, N, K, X.device)
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.bfloat16, device=X.device)
+    s_out = torch.empty((M,), dtype=torch.float32, device=X.device) if want_s_out else None
+    _check(lib().fpt_w4a4_linear_dynamic(_stream(), _ptr(X), M, K, _ptr(Wq), _ptr(sw), _scale_dtype(sw), N, bits, flags,
+                                         eps, _ptr(s_in), post_mode, _ptr(post), _ptr(Y), _ptr(s_out), _ptr(ws),
+                                         ws.numel()), "fpt_w4a4_linear_dynamic")
+    return Y, s_out

@@ -24,36 +24,6 @@ struct ActQuantParams {
   uint32_t flip;       // see quant_word
 };
 
-// acc + the 8 squares of a chunk in float64.  The bf16 magnitude bits, moved to the top of a
-// float64's high word, are the value times 2^-896 for every finite input (normal, subnormal or
-// zero alike); one exact multiply by 2^896 restores it, the square is exact in float64 and the
-// fused add rounds once.  Inf and NaN inputs come out as huge finite numbers here: the caller
-// recognises them by the overflowing float32 sum and redoes the row with sumsq_exact.
-__device__ __forceinline__ double sumsq(const uint4& v, double acc) {
-  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-  const double rebias = __hiloint2double(0x77F00000, 0);            // 2^896
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const double a = __hiloint2double((int)((w[i] & 0x7FFFu) << 13), 0) * rebias;
-    const double b = __hiloint2double((int)((w[i] >> 3) & 0x0FFFE000u), 0) * rebias;
-    acc = fma(a, a, acc);
-    acc = fma(b, b, acc);
-  }
-  return acc;
-}
-
-// The same sum by the definition (float32 square, widened, added): used for rows with Inf / NaN.
-__device__ __forceinline__ double sumsq_exact(const uint4& v, double acc) {
-  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const float a = bf16lo_to_f32(w[i]), b = bf16hi_to_f32(w[i]);
-    acc += (double)__fmul_rn(a, a);
-    acc += (double)__fmul_rn(b, b);
-  }
-  return acc;
-}
-
 // T threads per token, up to V 16-byte chunks (8 elements) per thread held in registers.
 template <int T, int V>
 __global__ void __launch_bounds__(T) act_quant_kernel(const ActQuantParams P) {

@@ -250,3 +250,29 @@ extern "C" int fpt_decoder_attn_out(void* stream, const void* A, int M, int k_o,
   return fpt_w4a4_gemm(stream, Aq, Wo_q, M, d, k_o, sw_o, scale_dtype, wsum_o, qp_ap->scale, qp_ap->symmetric,
                        qp_ap->zero_point, nullptr, X, X ? r : nullptr, Y, nullptr, workspace, gemm_ws);
 }
+
+extern "C" int fpt_w4a4_linear_dynamic(void* stream, const void* X, int M, int K, const uint8_t* Wq, const void* sw,
+                                       int scale_dtype, int N, int bits, int flags, float eps, const float* s_in,
+                                       int post_mode, const float* post, void* Y, float* s_out, void* workspace,
+                                       size_t workspace_bytes) {
+  if (!X || !Wq || !sw || !Y) return FPT_ERR_BAD_ARG;
+  if (bits != 4) return FPT_ERR_UNSUPPORTED;
+  int rc = check_gemm_shape(M, N, K);
+  if (rc) return rc;
+  if (flags & ~(FPT_RMSNORM | FPT_SCALE_INPUT)) return FPT_ERR_UNSUPPORTED;
+  if ((flags & FPT_SCALE_INPUT) && !s_in) return FPT_ERR_BAD_ARG;
+  if (post_mode < FPT_POST_NONE || post_mode > FPT_POST_VECTOR) return FPT_ERR_BAD_ARG;
+  if (post_mode == FPT_POST_VECTOR && !post) return FPT_ERR_BAD_ARG;
+  if (((uintptr_t)X | (uintptr_t)Wq | (uintptr_t)Y | (uintptr_t)workspace) & 15) return FPT_ERR_ALIGNMENT;
+  if (!workspace || workspace_bytes < fpt_workspace_bytes(FPT_OP_LINEAR, M, N, K)) return FPT_ERR_WORKSPACE;
+  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+  const size_t gemm_ws = kStatusBytes + gemm_scratch_bytes(M);
+  uint8_t* Xq = ws + gemm_ws;
+  float* c_t = reinterpret_cast<float*>(Xq + up256((size_t)M * K / 2));
+  // per-token grid; the factor the epilogue needs (D_t, times whatever the post mode asks for) per token
+  if (act_quant_dyn_launch((cudaStream_t)stream, X, M, K, K, 4, 1, 1.0f, flags, eps, s_in, post_mode, post, Xq, s_out,
+                           c_t, nullptr, nullptr) != cudaSuccess)
+    return FPT_ERR_CUDA;
+  return fpt_w4a4_gemm(stream, Xq, Wq, M, N, K, sw, scale_dtype, nullptr, 1.0f, 1, 0, c_t, nullptr, nullptr, Y, nullptr,
+                       workspace, gemm_ws);
+}

@@ -36,6 +36,11 @@ struct GemmParams {
 cudaError_t act_quant_launch(cudaStream_t st, const void* X, int M, int K, int ldx, const fpt_qparams* qp,
                              int flags, float eps, const void* X2, const float* s_in, uint8_t* Xq,
                              float* s_out, float* post_inv, float* r_out);
+// Dynamic (per-token grid) and 8-bit forms of the same step (act_quant_dynamic.cu).
+cudaError_t act_quant_dyn_launch(cudaStream_t st, const void* X, int M, int K, int ldx, int bits, int dynamic,
+                                 float qp_scale, int flags, float eps, const float* s_in, int post_mode,
+                                 const float* post, void* Xq, float* s_out, float* c_out, float* delta_out,
+                                 float* r_out);
 
 // hadamard_quant.cu: block-wise Hadamard + per-token scale + quantise (validated arguments only).
 int hadamard_block(int K);

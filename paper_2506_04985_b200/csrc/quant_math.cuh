@@ -50,11 +50,11 @@ __device__ __forceinline__ uint64_t mul_f32x2(uint64_t a, uint64_t b) {
   asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
   return r;
 }
-__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
-  uint64_t r;
-  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-  return r;
-}
+// (There is no packed add here on purpose.  The quantiser needs the product (x * p) * (1/D) ROUNDED
+// before the rounding constant is added; a packed multiply followed by a packed add was contracted
+// into one fused multiply-add -- the explicit .rn of the packed forms does not stop that -- and a
+// product that rounds to exactly k + 1/2 from slightly off it then took the other code.  The scalar
+// add intrinsic is never contracted.)
 
 // Quantiser arithmetic of one 16-byte chunk (8 values), in the order the header states:
 //   u = (x * p) * (1/D)          two separately rounded float32 multiplies
@@ -66,7 +66,7 @@ __device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
 // NaN at qmax - qmin = 15, i.e. the lowest code; the nibbles are flipped back by one XOR per
 // word (15 - c = c ^ 15; on the symmetric grid the two's complement nibble of 7 - c is c ^ 7).
 struct QuantConsts {
-  uint64_t np2, d2, m2;   // (-p, -p), (1/D, 1/D), (magic, magic)
+  uint64_t np2, d2;       // (-p, -p), (1/D, 1/D)
   int bias;               // -(bits of magic) + (qmax - z)
   uint32_t flip;          // 0x77777777 symmetric, 0xFFFFFFFF asymmetric
 };
@@ -77,7 +77,6 @@ __device__ __forceinline__ QuantConsts quant_consts(float p, float inv_delta, in
   QuantConsts c;
   c.np2 = pack_f32x2(-p, -p);
   c.d2 = pack_f32x2(inv_delta, inv_delta);
-  c.m2 = pack_f32x2(12582912.0f, 12582912.0f);
   c.bias = -0x4B400000 + qmax_minus_z;
   c.flip = flip;
   return c;
@@ -86,7 +85,9 @@ __device__ __forceinline__ QuantConsts quant_consts(float p, float inv_delta, in
 // Two values of one 32-bit word -> (15 - code) each, the second in front: returns c0 + 16 * c1 + 256 * prev.
 __device__ __forceinline__ uint32_t quant_pair(uint32_t w, const QuantConsts& c, uint32_t prev) {
   float v0, v1;
-  unpack_f32x2(add_f32x2(mul_f32x2(mul_f32x2(pack_f32x2(bf16lo_to_f32(w), bf16hi_to_f32(w)), c.np2), c.d2), c.m2), v0, v1);
+  unpack_f32x2(mul_f32x2(mul_f32x2(pack_f32x2(bf16lo_to_f32(w), bf16hi_to_f32(w)), c.np2), c.d2), v0, v1);
+  v0 = __fadd_rn(v0, 12582912.0f);
+  v1 = __fadd_rn(v1, 12582912.0f);
   // (a negative sum -- u beyond 1.2e7 -- has a negative pattern; max(., 0) keeps the add below from wrapping)
   const uint32_t c0 = (uint32_t)__viaddmin_s32_relu(max(__float_as_int(v0), 0), c.bias, 15);
   const uint32_t c1 = (uint32_t)__viaddmin_s32_relu(max(__float_as_int(v1), 0), c.bias, 15);
@@ -96,7 +97,9 @@ __device__ __forceinline__ uint32_t quant_pair(uint32_t w, const QuantConsts& c,
 // The same for two float32 values (no 16-bit rounding in front of the grid).
 __device__ __forceinline__ uint32_t quant_pair_f32(float x0, float x1, const QuantConsts& c, uint32_t prev) {
   float v0, v1;
-  unpack_f32x2(add_f32x2(mul_f32x2(mul_f32x2(pack_f32x2(x0, x1), c.np2), c.d2), c.m2), v0, v1);
+  unpack_f32x2(mul_f32x2(mul_f32x2(pack_f32x2(x0, x1), c.np2), c.d2), v0, v1);
+  v0 = __fadd_rn(v0, 12582912.0f);
+  v1 = __fadd_rn(v1, 12582912.0f);
   const uint32_t c0 = (uint32_t)__viaddmin_s32_relu(max(__float_as_int(v0), 0), c.bias, 15);
   const uint32_t c1 = (uint32_t)__viaddmin_s32_relu(max(__float_as_int(v1), 0), c.bias, 15);
   return (prev * 16u + c1) * 16u + c0;
@@ -117,6 +120,36 @@ __device__ __forceinline__ uint32_t quant_word(const uint4& v, const QuantConsts
   w = quant_pair(v.y, c, w);
   w = quant_pair(v.x, c, w);
   return w ^ c.flip;
+}
+
+// acc + the 8 squares of a chunk in float64.  The bf16 magnitude bits, moved to the top of a
+// float64's high word, are the value times 2^-896 for every finite input (normal, subnormal or
+// zero alike); one exact multiply by 2^896 restores it, the square is exact in float64 and the
+// fused add rounds once.  Inf and NaN inputs come out as huge finite numbers here: the caller
+// recognises them by the overflowing float32 sum and redoes the row with sumsq_exact.
+__device__ __forceinline__ double sumsq(const uint4& v, double acc) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+  const double rebias = __hiloint2double(0x77F00000, 0);            // 2^896
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const double a = __hiloint2double((int)((w[i] & 0x7FFFu) << 13), 0) * rebias;
+    const double b = __hiloint2double((int)((w[i] >> 3) & 0x0FFFE000u), 0) * rebias;
+    acc = fma(a, a, acc);
+    acc = fma(b, b, acc);
+  }
+  return acc;
+}
+
+// The same sum by the definition (float32 square, widened, added): used for rows with Inf / NaN.
+__device__ __forceinline__ double sumsq_exact(const uint4& v, double acc) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float a = bf16lo_to_f32(w[i]), b = bf16hi_to_f32(w[i]);
+    acc += (double)__fmul_rn(a, a);
+    acc += (double)__fmul_rn(b, b);
+  }
+  return acc;
 }
 
 }  // namespace fpt

@@ -127,3 +127,47 @@ def test_interleave_gate_up_layout():
         assert np.array_equal(wgu[128 * r + 64:128 * r + 128], u[64 * r:64 * r + 64].numpy())
         assert np.array_equal(sw[128 * r:128 * r + 64], sg[64 * r:64 * r + 64].numpy())
         assert np.array_equal(sw[128 * r + 64:128 * r + 128], su[64 * r:64 * r + 64].numpy())
+
+
+def _rows_with_products_that_round_to_a_tie(scale, n_rows, K, seed):
+    """Per-token multipliers p and bf16 inputs for which (x * p) * (1/D) is exactly k + 1/2 after its
+    two roundings while the unrounded product is not: a kernel that contracts the second multiply
+    with anything that follows takes the other code there.  Found by search over all bf16 values."""
+    rng = np.random.default_rng(seed)
+    F = np.float32
+    inv = F(1.0) / F(scale)
+    vals = np.arange(0x3C00, 0x4300, dtype=np.uint32)                       # bf16 patterns of about 0.008 .. 128
+    xs = (vals << 16).view(F)
+    rows, ps, hits = [], [], 0
+    while len(rows) < n_rows:
+        cand = np.exp(rng.uniform(-3.0, 0.5, 4096)).astype(F)                # many multipliers at once
+        v = (xs[None, :] * cand[:, None]).astype(F)
+        u = (v * inv).astype(F)
+        tie = (np.abs(u) < 8) & (u - np.floor(u) == F(0.5))
+        off = v.astype(np.float64) * np.float64(inv) != u.astype(np.float64)
+        good = tie & off
+        for i in np.nonzero(good.any(axis=1))[0]:
+            if len(rows) == n_rows:
+                break
+            sel = xs[good[i]]
+            row = rng.choice(xs, K).astype(F) * rng.choice([-1, 1], K).astype(F)
+            row[:sel.size] = sel
+            row[sel.size:2 * sel.size] = -sel
+            hits += 2 * sel.size
+            rows.append(row)
+            ps.append(cand[i])
+    return np.stack(rows), np.array(ps, dtype=F), hits
+
+
+@pytest.mark.parametrize("K", [256, 4096])
+def test_act_quant_products_that_round_to_a_tie(K):
+    scale = 0.62
+    x, p, hits = _rows_with_products_that_round_to_a_tie(scale, 60, K, 9)
+    assert hits >= 100
+    x, p = np.tile(x, (10, 1)), np.tile(p, 10)           # 600 tokens: enough for the many-token kernels
+    xb = synth.to_bf16(x)
+    qp = B.QParams(4, True, scale, 0)
+    for M in (600, 24):                                  # the many-token and the few-token kernels
+        xq, _ = B.fpt_act_quant(dev(xb[:M]), qp, B.SCALE_INPUT, 0.0, s_in=dev(torch.from_numpy(p[:M])))
+        codes, _, _, _ = OQ.act_quant(synth.f32(xb[:M]), oqp(qp), False, True, 0.0, p[:M])
+        assert np.array_equal(host(xq), OQ.pack_int4(codes))
