@@ -76,11 +76,13 @@ extern "C" {
 #define FPT_OP_LINEAR 0
 #define FPT_OP_MLP    1
 #define FPT_OP_GEMM   2
+#define FPT_OP_GEMM_A8   3     /* fpt_w4a8_gemm                                   */
+#define FPT_OP_LINEAR_A8 4     /* fpt_w4a4_linear / _dynamic with 8-bit activations */
 
 /* One quantiser, as the paper parametrises it: bit-width, grid kind, static scale and
  * offset (App. D "General set-up"). HOST struct. */
 typedef struct fpt_qparams {
-  int   bits;        /* 4 */
+  int   bits;        /* 4; 8 for activations where an entry point says so (symmetric only) */
   int   symmetric;   /* 1: codes in [-8, 7], zero_point ignored; 0: codes in [0, 15]     */
   float scale;       /* static per-tensor scale D (activations); ignored for weights,    */
                      /* whose per-output-channel scales are computed                     */
@@ -137,7 +139,8 @@ int fpt_interleave_gate_up(void* stream, const uint8_t* Wg_q, const uint8_t* Wu_
  *          ignored, X is [M, 2K] (ldx >= 2K) and logical column k lives at
  *          gate: (k/64)*128 + k%64, up: gate + 64
  *   s_in   [M] f32 or NULL;  s_out [M] f32 or NULL
- *   Xq     [M, K/2] packed codes out
+ *   Xq     [M, K/2] packed codes out;  qp->bits == 8 (symmetric grid, no FPT_SILU_MUL): [M, K] int8 codes
+ *          q = clamp(rne((x * p) * (1/D)), -128, 127)
  * silu(g) = g / (1 + 2^(-g*log2 e)) with a fixed float32 polynomial for 2^f (degree 6
  * Taylor, Horner, separately rounded multiply and add), so that the result is one
  * defined float32 value.
@@ -203,11 +206,28 @@ int fpt_w4a4_gemm(void* stream, const uint8_t* Xq, const uint8_t* Wq, int M, int
                   void* Y, int32_t* acc_out, void* workspace, size_t workspace_bytes);
 
 /*
+ * The same two steps with 8-bit activation codes and 4-bit weights (the W4A8 setting, Sec. 4):
+ *   acc[t,n] = sum_k qa[t,k] * qw[n,k]      exact int32;  qa int8 in [-128, 127] (symmetric grid)
+ *   y[t,n]   as in fpt_w4a4_gemm.
+ *   Xq8 [M, K] int8;  K % 128 == 0, K <= 16384 (so that (float)acc is exact), N % 8 == 0.
+ *   workspace: fpt_workspace_bytes(FPT_OP_GEMM_A8, M, N, K) bytes.
+ * More than 128 tokens and 128 outputs: one matmul kernel that loads the activation tile as int8.
+ * Smaller problems: the codes are split as a = 16 (a >> 4) + (a & 15) and two 4-bit matmuls are
+ * combined exactly in int32 before the scale factors (same result, twice the matmul work).
+ */
+int fpt_w4a8_gemm(void* stream, const int8_t* Xq8, const uint8_t* Wq, int M, int N, int K,
+                  const void* sw, int scale_dtype, float act_scale,
+                  const float* post, const void* residual, const float* res_scale,
+                  void* Y, int32_t* acc_out, void* workspace, size_t workspace_bytes);
+
+/*
  * Steps (1)+(2)+(3): one W4A4 linear on bf16 activations.
  *   X [M, K] bf16; flags / eps / s_in / s_out as in fpt_act_quant (FPT_SILU_MUL not allowed);
  *   post_mode selects c_t (see FPT_POST_*); post [M] only for FPT_POST_VECTOR.
  *   workspace: fpt_workspace_bytes(FPT_OP_LINEAR, M, N, K) bytes (packed activations,
  *   the per-token vectors and the status word live there).
+ * act_qp->bits == 8 (symmetric grid only): int8 codes q = clamp(rne((x * p) * (1/D)), -128, 127) and
+ *   the matmul of fpt_w4a8_gemm; workspace: fpt_workspace_bytes(FPT_OP_LINEAR_A8, M, N, K) bytes.
  */
 int fpt_w4a4_linear(void* stream, const void* X, int M, int K,
                     const uint8_t* Wq, const void* sw, int scale_dtype, const int32_t* wsum, int N,
@@ -221,7 +241,8 @@ int fpt_w4a4_linear(void* stream, const void* X, int M, int K,
  *   codes, D_t as in fpt_act_quant_dynamic;  acc as in fpt_w4a4_gemm (symmetric codes);
  *   y[t,n] = bf16( ((float)acc * sw[n]) * c_t ),
  *   c_t = D_t (FPT_POST_NONE), D_t * (1 / p_t) (FPT_POST_INVERSE_OF_PRE), D_t * post[t] (FPT_POST_VECTOR).
- *   bits = 4 in this version.  workspace: fpt_workspace_bytes(FPT_OP_LINEAR, M, N, K) bytes.
+ *   bits = 4: workspace fpt_workspace_bytes(FPT_OP_LINEAR, M, N, K) bytes;
+ *   bits = 8: int8 codes, matmul of fpt_w4a8_gemm, workspace fpt_workspace_bytes(FPT_OP_LINEAR_A8, M, N, K).
  */
 int fpt_w4a4_linear_dynamic(void* stream, const void* X, int M, int K,
                             const uint8_t* Wq, const void* sw, int scale_dtype, int N,
@@ -313,7 +334,7 @@ int fpt_decoder_attn_out(void* stream, const void* A, int M, int k_o,
                          void* Y, void* workspace, size_t workspace_bytes);
 
 /* Bytes of caller-provided scratch an entry point needs (op = FPT_OP_*).
- * FPT_OP_LINEAR / FPT_OP_GEMM: (M, N, K); FPT_OP_MLP: (M, d_ff, d). */
+ * FPT_OP_LINEAR / FPT_OP_GEMM / FPT_OP_GEMM_A8 / FPT_OP_LINEAR_A8: (M, N, K); FPT_OP_MLP: (M, d_ff, d). */
 size_t fpt_workspace_bytes(int op, int M, int N, int K);
 
 /* Zeroes the control block (first 8 KiB: status word, tile counters) of a workspace.  Call once

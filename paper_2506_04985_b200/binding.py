@@ -19,11 +19,11 @@ DTYPE_BF16, DTYPE_F32, DTYPE_F16 = 0, 1, 2
 RANGE_MINMAX, RANGE_LP = 0, 1
 RMSNORM, SCALE_INPUT, SILU_MUL, GU_INTERLEAVED = 1, 2, 4, 8
 POST_NONE, POST_INVERSE_OF_PRE, POST_VECTOR = 0, 1, 2
-OP_LINEAR, OP_MLP, OP_GEMM = 0, 1, 2
+OP_LINEAR, OP_MLP, OP_GEMM, OP_GEMM_A8, OP_LINEAR_A8 = 0, 1, 2, 3, 4
 
 EXPORTS = ["fpt_version", "fpt_strerror", "fpt_quantize_weights", "fpt_interleave_gate_up", "fpt_act_quant", "fpt_hadamard_quant",
            "fpt_w4a4_gemm", "fpt_w4a4_linear", "fpt_w4a4_linear_static", "fpt_decoder_mlp", "fpt_decoder_attn_qkv",
-           "fpt_decoder_attn_out", "fpt_act_quant_dynamic", "fpt_w4a4_linear_dynamic", "fpt_workspace_bytes",
+           "fpt_decoder_attn_out", "fpt_act_quant_dynamic", "fpt_w4a4_linear_dynamic", "fpt_w4a8_gemm", "fpt_workspace_bytes",
            "fpt_reset_status",
            "fpt_check_status"]
 
@@ -66,6 +66,7 @@ def lib():
         L.fpt_w4a4_linear_static.argtypes = [vp, vp, ci, ci, vp, vp, ci, vp, ci, qp, ci, cf, vp, ci, vp, vp, vp]
         L.fpt_decoder_mlp.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp, vp, ci, qp, qp, cf, vp, vp, ci, ci, vp, vp, sz]
         L.fpt_hadamard_quant.argtypes = [vp, vp, ci, ci, ci, qp, ci, vp, vp]
+        L.fpt_w4a8_gemm.argtypes = [vp, vp, vp, ci, ci, ci, vp, ci, cf, vp, vp, vp, vp, vp, vp, sz]
         L.fpt_act_quant_dynamic.argtypes = [vp, vp, ci, ci, ci, ci, ci, cf, vp, vp, vp, vp]
         L.fpt_w4a4_linear_dynamic.argtypes = [vp, vp, ci, ci, vp, vp, ci, ci, ci, ci, cf, vp, ci, vp, vp, vp, vp, sz]
         L.fpt_decoder_attn_qkv.argtypes = [vp, vp, ci, ci, vp, vp, ci, vp, ci, qp, cf, vp, vp, vp, vp, vp, sz]
@@ -149,7 +150,12 @@ def fpt_act_quant(X, qp, flags=RMSNORM, eps=1e-5, X2=None, s_in=None, K=None, wa
     M, ldx = X.shape
     if K is None:
         K = ldx // 2 if (flags & GU_INTERLEAVED) else ldx
-    Xq = out if out is not None else torch.empty((M, K // 2), dtype=torch.uint8, device=X.device)
+    if out is not None:
+        Xq = out
+    elif qp.bits == 8:
+        Xq = torch.empty((M, K), dtype=torch.int8, device=X.device)
+    else:
+        Xq = torch.empty((M, K // 2), dtype=torch.uint8, device=X.device)
     s_out = torch.empty((M,), dtype=torch.float32, device=X.device) if want_s_out else None
     _check(lib().fpt_act_quant(_stream(), _ptr(X), M, K, ldx, ctypes.byref(qp), flags, eps, _ptr(X2), _ptr(s_in),
                                _ptr(Xq), _ptr(s_out)), "fpt_act_quant")
@@ -180,7 +186,7 @@ def fpt_w4a4_linear(X, Wq, sw, qp, flags=RMSNORM, eps=1e-5, s_in=None, post_mode
     M, K = X.shape
     N = Wq.shape[0]
     if ws is None:
-        ws = new_workspace(OP_LINEAR, M, N, K, X.device)
+        ws = new_workspace(OP_LINEAR_A8 if qp.bits == 8 else OP_LINEAR, M, N, K, X.device)
     if Y is None:
         Y = torch.empty((M, N), dtype=torch.bfloat16, device=X.device)
     s_out = torch.empty((M,), dtype=torch.float32, device=X.device) if want_s_out else None
@@ -286,7 +292,7 @@ def fpt_w4a4_linear_dynamic(X, Wq, sw, bits=4, flags=RMSNORM, eps=1e-5, s_in=Non
     M, K = X.shape
     N = Wq.shape[0]
     if ws is None:
-        ws = new_workspace(OP_LINEAR, M, N, K, X.device)
+        ws = new_workspace(OP_LINEAR_A8 if bits == 8 else OP_LINEAR, M, N, K, X.device)
     if Y is None:
         Y = torch.empty((M, N), dtype=torch.bfloat16, device=X.device)
     s_out = torch.empty((M,), dtype=torch.float32, device=X.device) if want_s_out else None
@@ -294,3 +300,19 @@ def fpt_w4a4_linear_dynamic(X, Wq, sw, bits=4, flags=RMSNORM, eps=1e-5, s_in=Non
                                          eps, _ptr(s_in), post_mode, _ptr(post), _ptr(Y), _ptr(s_out), _ptr(ws),
                                          ws.numel()), "fpt_w4a4_linear_dynamic")
     return Y, s_out
+
+
+def fpt_w4a8_gemm(Xq8, Wq, sw, act_scale, post=None, residual=None, res_scale=None, want_y=True, want_acc=False,
+                  ws=None, Y=None):
+    """int8 [M, K] x packed 4-bit [N, K/2] matmul + scale factors -> (Y bf16 or None, acc int32 or None)."""
+    M, K = Xq8.shape
+    N = Wq.shape[0]
+    if ws is None:
+        ws = new_workspace(OP_GEMM_A8, M, N, K, Xq8.device)
+    if Y is None and want_y:
+        Y = torch.empty((M, N), dtype=torch.bfloat16, device=Xq8.device)
+    acc = torch.empty((M, N), dtype=torch.int32, device=Xq8.device) if want_acc else None
+    _check(lib().fpt_w4a8_gemm(_stream(), _ptr(Xq8), _ptr(Wq), M, N, K, _ptr(sw), _scale_dtype(sw), float(act_scale),
+                               _ptr(post), _ptr(residual), _ptr(res_scale), _ptr(Y), _ptr(acc), _ptr(ws), ws.numel()),
+           "fpt_w4a8_gemm")
+    return Y, acc

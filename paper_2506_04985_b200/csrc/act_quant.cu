@@ -349,6 +349,15 @@ extern "C" int fpt_act_quant(void* stream, const void* X, int M, int K, int ldx,
                              int flags, float eps, const void* X2, const float* s_in, uint8_t* Xq,
                              float* s_out) {
   if (!X || !qp || !Xq || M <= 0 || K <= 0) return FPT_ERR_BAD_ARG;
+  if (qp->bits == 8) {          // int8 codes [M, K] on the symmetric grid (W4A8); Xq then has K bytes per row
+    if (!qp->symmetric || (flags & ~(FPT_RMSNORM | FPT_SCALE_INPUT))) return FPT_ERR_UNSUPPORTED;
+    if (!(qp->scale > 0.0f) || ((flags & FPT_SCALE_INPUT) && !s_in)) return FPT_ERR_BAD_ARG;
+    if (K % 32 != 0 || K > 65536) return FPT_ERR_UNSUPPORTED;
+    if (ldx < K || ldx % 8 != 0 || (((uintptr_t)X | (uintptr_t)Xq) & 15)) return FPT_ERR_ALIGNMENT;
+    cudaError_t e8 = fpt::act_quant_dyn_launch((cudaStream_t)stream, X, M, K, ldx, 8, 0, qp->scale, flags, eps, s_in,
+                                               FPT_POST_NONE, nullptr, Xq, s_out, nullptr, nullptr, nullptr);
+    return e8 == cudaSuccess ? FPT_OK : FPT_ERR_CUDA;
+  }
   if (qp->bits != 4) return FPT_ERR_UNSUPPORTED;
   if (!(qp->scale > 0.0f)) return FPT_ERR_BAD_ARG;
   if (!qp->symmetric && (qp->zero_point < 0 || qp->zero_point > 15)) return FPT_ERR_BAD_ARG;

@@ -47,6 +47,10 @@ extern "C" size_t fpt_workspace_bytes(int op, int M, int N, int K) {
       return kStatusBytes + gemm_scratch_bytes(M);
     case FPT_OP_LINEAR:
       return kStatusBytes + gemm_scratch_bytes(M) + up256(m * (size_t)K / 2) + up256(m * 4);
+    case FPT_OP_GEMM_A8:
+      return kStatusBytes + gemm_scratch_bytes(M) + gemm_a8_scratch_bytes(M, N, K);
+    case FPT_OP_LINEAR_A8:
+      return kStatusBytes + gemm_scratch_bytes(M) + gemm_a8_scratch_bytes(M, N, K) + up256(m * (size_t)K) + up256(m * 4);
     case FPT_OP_MLP: {   // N = d_ff, K = d
       const size_t dff = (size_t)N, d = (size_t)K;
       return kStatusBytes + gemm_scratch_bytes(M) + up256(m * d / 2) + 2 * up256(m * 4) + up256(m * 2 * dff * 2) +
@@ -107,7 +111,8 @@ extern "C" int fpt_w4a4_linear(void* stream, const void* X, int M, int K, const 
                                float eps, const float* s_in, int post_mode, const float* post, void* Y, float* s_out,
                                void* workspace, size_t workspace_bytes) {
   if (!X || !Wq || !sw || !Y) return FPT_ERR_BAD_ARG;
-  int rc = check_qp(act_qp);
+  const bool a8 = act_qp && act_qp->bits == 8;
+  int rc = a8 ? ((act_qp->symmetric && act_qp->scale > 0.0f) ? FPT_OK : FPT_ERR_UNSUPPORTED) : check_qp(act_qp);
   if (rc) return rc;
   rc = check_gemm_shape(M, N, K);
   if (rc) return rc;
@@ -115,6 +120,20 @@ extern "C" int fpt_w4a4_linear(void* stream, const void* X, int M, int K, const 
   if ((flags & FPT_SCALE_INPUT) && !s_in) return FPT_ERR_BAD_ARG;
   if (post_mode < FPT_POST_NONE || post_mode > FPT_POST_VECTOR) return FPT_ERR_BAD_ARG;
   if (post_mode == FPT_POST_VECTOR && !post) return FPT_ERR_BAD_ARG;
+  if (a8) {
+    if (((uintptr_t)X | (uintptr_t)Wq | (uintptr_t)Y | (uintptr_t)workspace) & 15) return FPT_ERR_ALIGNMENT;
+    if (!workspace || workspace_bytes < fpt_workspace_bytes(FPT_OP_LINEAR_A8, M, N, K)) return FPT_ERR_WORKSPACE;
+    const size_t gemm_ws8 = fpt_workspace_bytes(FPT_OP_GEMM_A8, M, N, K);
+    int8_t* Xq8 = reinterpret_cast<int8_t*>(workspace) + gemm_ws8;
+    float* pinv = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(Xq8) + up256((size_t)M * K));
+    if (act_quant_dyn_launch((cudaStream_t)stream, X, M, K, K, 8, 0, act_qp->scale, flags, eps, s_in, post_mode, post,
+                             Xq8, s_out, post_mode == FPT_POST_INVERSE_OF_PRE ? pinv : nullptr, nullptr,
+                             nullptr) != cudaSuccess)
+      return FPT_ERR_CUDA;
+    const float* pv8 = post_mode == FPT_POST_NONE ? nullptr : post_mode == FPT_POST_VECTOR ? post : pinv;
+    return fpt_w4a8_gemm(stream, Xq8, Wq, M, N, K, sw, scale_dtype, act_qp->scale, pv8, nullptr, nullptr, Y, nullptr,
+                         workspace, gemm_ws8);
+  }
   if (!act_qp->symmetric && !wsum) return FPT_ERR_BAD_ARG;
   if (((uintptr_t)X | (uintptr_t)Wq | (uintptr_t)Y | (uintptr_t)workspace) & 15) return FPT_ERR_ALIGNMENT;
   if (!workspace || workspace_bytes < fpt_workspace_bytes(FPT_OP_LINEAR, M, N, K)) return FPT_ERR_WORKSPACE;
@@ -256,7 +275,7 @@ extern "C" int fpt_w4a4_linear_dynamic(void* stream, const void* X, int M, int K
                                        int post_mode, const float* post, void* Y, float* s_out, void* workspace,
                                        size_t workspace_bytes) {
   if (!X || !Wq || !sw || !Y) return FPT_ERR_BAD_ARG;
-  if (bits != 4) return FPT_ERR_UNSUPPORTED;
+  if (bits != 4 && bits != 8) return FPT_ERR_UNSUPPORTED;
   int rc = check_gemm_shape(M, N, K);
   if (rc) return rc;
   if (flags & ~(FPT_RMSNORM | FPT_SCALE_INPUT)) return FPT_ERR_UNSUPPORTED;
@@ -264,6 +283,17 @@ extern "C" int fpt_w4a4_linear_dynamic(void* stream, const void* X, int M, int K
   if (post_mode < FPT_POST_NONE || post_mode > FPT_POST_VECTOR) return FPT_ERR_BAD_ARG;
   if (post_mode == FPT_POST_VECTOR && !post) return FPT_ERR_BAD_ARG;
   if (((uintptr_t)X | (uintptr_t)Wq | (uintptr_t)Y | (uintptr_t)workspace) & 15) return FPT_ERR_ALIGNMENT;
+  if (bits == 8) {
+    if (!workspace || workspace_bytes < fpt_workspace_bytes(FPT_OP_LINEAR_A8, M, N, K)) return FPT_ERR_WORKSPACE;
+    const size_t gemm_ws8 = fpt_workspace_bytes(FPT_OP_GEMM_A8, M, N, K);
+    int8_t* Xq8 = reinterpret_cast<int8_t*>(workspace) + gemm_ws8;
+    float* c8 = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(Xq8) + up256((size_t)M * K));
+    if (act_quant_dyn_launch((cudaStream_t)stream, X, M, K, K, 8, 1, 1.0f, flags, eps, s_in, post_mode, post, Xq8, s_out,
+                             c8, nullptr, nullptr) != cudaSuccess)
+      return FPT_ERR_CUDA;
+    return fpt_w4a8_gemm(stream, Xq8, Wq, M, N, K, sw, scale_dtype, 1.0f, c8, nullptr, nullptr, Y, nullptr, workspace,
+                         gemm_ws8);
+  }
   if (!workspace || workspace_bytes < fpt_workspace_bytes(FPT_OP_LINEAR, M, N, K)) return FPT_ERR_WORKSPACE;
   uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
   const size_t gemm_ws = kStatusBytes + gemm_scratch_bytes(M);

@@ -13,6 +13,7 @@ struct GemmParams {
   const int32_t* wsum;
   int zero_point;              // 0 when the activation grid is symmetric
   int a_unsigned;              // activation codes are unsigned nibbles (asymmetric grid)
+  int a_bits;                  // 8: the activation operand is int8 [M, K] (CTA-pair kernel only); otherwise packed 4-bit
   float act_scale;
   const float* post;
   const __nv_bfloat16* residual;
@@ -31,6 +32,9 @@ struct GemmParams {
   uint32_t* status;            // control block of the workspace (status word, decode counters)
   void* scratch;               // gemm_scratch_bytes(M) bytes behind the control block (decode partial sums)
 };
+
+// gemm_a8.cu: scratch bytes fpt_w4a8_gemm needs behind the control block and the matmul scratch.
+size_t gemm_a8_scratch_bytes(int M, int N, int K);
 
 // act_quant.cu: validated arguments only; also fills 1/p_t and r_t for the composed calls.
 cudaError_t act_quant_launch(cudaStream_t st, const void* X, int M, int K, int ldx, const fpt_qparams* qp,

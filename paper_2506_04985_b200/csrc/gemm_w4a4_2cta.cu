@@ -42,14 +42,17 @@ constexpr int kConvAWarp0 = 4, kConvBWarp0 = 8, kEpiWarp0 = 12, kEpiWarps = 8;
 
 // NS: stages of widened operands (int8 weight tile in shared memory + activation columns in
 // tensor memory); NPK: stages of packed tiles in flight from TMA.
-template <int NS, int NPK>
+// kA8: the activation operand arrives as int8 codes (one byte each, 128-byte rows per k-block)
+// instead of packed 4-bit codes.
+template <int NS, int NPK, bool kA8 = false>
 struct Smem {
   static_assert(kAccCols + NS * kAStageCols <= kTmemCols, "operand stages must fit beside the accumulator");
   static constexpr int kB8Stage = HR * I8_ROW;                      // 16 KB
-  static constexpr int kPkOp = HR * PK_ROW;                         // 8 KB
+  static constexpr int kPkOp = HR * PK_ROW;                         // 8 KB: a packed weight tile
+  static constexpr int kPkOpA = kA8 ? HR * I8_ROW : HR * PK_ROW;    // the activation tile of a stage
   static constexpr int kB8Off = 0;
   static constexpr int kPkAOff = kB8Off + NS * kB8Stage;
-  static constexpr int kPkBOff = kPkAOff + NPK * kPkOp;
+  static constexpr int kPkBOff = kPkAOff + NPK * kPkOpA;
   static constexpr int kStgOff = kPkBOff + NPK * kPkOp;             // bf16 output tile: 4 slabs of 128 rows x 64 columns
   static constexpr int kStgSlab = HR * 128;                         // 16 KB, 128-byte rows, 128-byte swizzle
   static constexpr int kScaleOff = kStgOff + 4 * kStgSlab;          // 2 x 256 floats (sw) + 2 x 256 ints (z * wsum)
@@ -83,11 +86,12 @@ __device__ __forceinline__ void load_scales8(const void* sw, int scale_dtype, in
 
 // kFuse: 0 plain scale-factor epilogue; 1 SwiGLU product + quantiser (codes out); 2 SwiGLU product
 // (bf16 out).  Separate instantiations keep the plain epilogue's register budget free of the others.
-template <int NS, int NPK, int kFuse>
+template <int NS, int NPK, int kFuse, bool kA8 = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                       const __grid_constant__ CUtensorMap tmY, const GemmParams P) {
-  using L = Smem<NS, NPK>;
+  using L = Smem<NS, NPK, kA8>;
+  static_assert(!kA8 || kFuse == 0, "8-bit activations: plain epilogue only");
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(smem);
@@ -149,8 +153,8 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         const int n0 = (tile / P.tiles_m) * TN + (int)rank * HR;
         for (int kb = 0; kb < P.kblocks; ++kb) {
           if (!mbar_wait(pk_empty(s), ph ^ 1u, abort_flag, P.status, 1)) { ok = false; break; }
-          mbar_arrive_expect_tx(pk_full(s), 2 * L::kPkOp);
-          tma_load_2d(sbase + L::kPkAOff + s * L::kPkOp, &tmA, pk_full(s), kb * PK_ROW, m0);
+          mbar_arrive_expect_tx(pk_full(s), L::kPkOpA + L::kPkOp);
+          tma_load_2d(sbase + L::kPkAOff + s * L::kPkOpA, &tmA, pk_full(s), kb * (kA8 ? I8_ROW : PK_ROW), m0);
           tma_load_2d(sbase + L::kPkBOff + s * L::kPkOp, &tmB, pk_full(s), kb * PK_ROW, n0);
           armed |= 1u << s;
           armed_par = (armed_par & ~(1u << s)) | (ph << s);
@@ -202,13 +206,31 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     for (int tile = pair_id; ok && tile < P.num_tiles; tile += num_pairs) {
       for (int kb = 0; kb < P.kblocks; ++kb) {
         if (!mbar_wait(pk_full(ps), pph, abort_flag, P.status, 5)) { ok = false; break; }
-        const uint8_t* src = smem + L::kPkAOff + ps * L::kPkOp + r * PK_ROW;
-        uint4 c[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) c[j] = *reinterpret_cast<const uint4*>(src + (((uint32_t)j ^ swz) << 4));
         uint32_t v[32];
+        if constexpr (kA8) {
+          // int8 codes, 128-byte rows under the 128-byte swizzle.  The weight side orders the 32 codes
+          // of a group as 16 even-k then 16 odd-k bytes (that is how the nibbles fall apart); the
+          // activation bytes are put into the same order.
+          const uint8_t* src = smem + L::kPkAOff + ps * L::kPkOpA + r * I8_ROW;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) widen(c[j], v + 8 * j);
+          for (int g = 0; g < 4; ++g) {
+            const uint4 c0 = *reinterpret_cast<const uint4*>(src + (((uint32_t)(2 * g) ^ (uint32_t)(r & 7)) << 4));
+            const uint4 c1 = *reinterpret_cast<const uint4*>(src + (((uint32_t)(2 * g + 1) ^ (uint32_t)(r & 7)) << 4));
+            const uint32_t a[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+#pragma unroll
+            for (int w = 0; w < 4; ++w) {
+              v[8 * g + w] = __byte_perm(a[2 * w], a[2 * w + 1], 0x6420);
+              v[8 * g + 4 + w] = __byte_perm(a[2 * w], a[2 * w + 1], 0x7531);
+            }
+          }
+        } else {
+          const uint8_t* src = smem + L::kPkAOff + ps * L::kPkOpA + r * PK_ROW;
+          uint4 c[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) c[j] = *reinterpret_cast<const uint4*>(src + (((uint32_t)j ^ swz) << 4));
+#pragma unroll
+          for (int j = 0; j < 4; ++j) widen(c[j], v + 8 * j);
+        }
         if (!mbar_wait(op_empty(s), ph ^ 1u, abort_flag, P.status, 6)) { ok = false; break; }
         tc_fence_after();
         tmem_st_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + kAccCols + s * kAStageCols, v);
@@ -271,7 +293,8 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     float* sw_s = reinterpret_cast<float*>(smem + L::kScaleOff);
     int* zw_s = reinterpret_cast<int*>(smem + L::kScaleOff + 2 * TN * 4);
     const int r = quad * 32 + lane;                      // row of the CTA's 128
-    const bool magic_ok = P.K <= 32768;                  // |acc| < 2^22: int -> float by exponent trick
+    constexpr int kShift = kA8 ? 4 : 8;                  // both operands carry a factor 16, int8 activations none
+    const bool magic_ok = kA8 ? P.K < 4096 : P.K <= 32768;   // |acc| < 2^22: int -> float by exponent trick
     const bool issuer = quad == 0 && lane == 0;          // issues the TMA stores of its half
     int it = 0;
     for (int tile = pair_id; tile < P.num_tiles; tile += num_pairs, ++it) {
@@ -351,7 +374,7 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
           const int col = nt + half * 128 + ch * 32 + g * 8;
           int a[8];
 #pragma unroll
-          for (int j = 0; j < 8; ++j) a[j] = (((int)v[ch * 32 + g * 8 + j]) >> 8) - zws[ch * 32 + g * 8 + j];
+          for (int j = 0; j < 8; ++j) a[j] = (((int)v[ch * 32 + g * 8 + j]) >> kShift) - zws[ch * 32 + g * 8 + j];
           if (P.acc_out && row_ok && col < P.N) {
             int4* o = reinterpret_cast<int4*>(P.acc_out + rowoff + col);
             o[0] = make_int4(a[0], a[1], a[2], a[3]);
@@ -454,6 +477,19 @@ static bool make_map(CUtensorMap* m, const void* base, int rows, int K, CUtensor
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tensor map over an int8 [rows, K]-byte matrix; one box = 128 rows of one k-block (128 bytes each).
+static bool make_map_i8(CUtensorMap* m, const void* base, int rows, int K) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)K};
+  const cuuint32_t box[2] = {(cuuint32_t)I8_ROW, (cuuint32_t)HR};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // Tensor map over the bf16 output [M, N]; one box = 128 rows x 64 columns, 128-byte swizzle in shared memory.
 static bool make_out_map(CUtensorMap* m, const void* base, int M, int N) {
   EncodeTiledFn fn = encode_fn();
@@ -480,10 +516,10 @@ static bool make_codes_map(CUtensorMap* m, const void* base, int M, int row_byte
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int NS, int NPK, int kFuse>
+template <int NS, int NPK, int kFuse, bool kA8 = false>
 static int launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, GemmParams P) {
-  using L = Smem<NS, NPK>;
-  auto kern = gemm_w4a4_pair_kernel<NS, NPK, kFuse>;
+  using L = Smem<NS, NPK, kA8>;
+  auto kern = gemm_w4a4_pair_kernel<NS, NPK, kFuse, kA8>;
   static int max_pairs = 0;                 // co-resident CTA pairs on this device
   if (!max_pairs) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kAlloc) != cudaSuccess)
@@ -507,7 +543,8 @@ static int launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, GemmPar
     max_pairs = n > 0 ? n : 1;
   }
   CUtensorMap tmA, tmB, tmY;
-  if (!make_map(&tmA, Xq, P.M, P.K, CU_TENSOR_MAP_SWIZZLE_64B) || !make_map(&tmB, Wq, P.N, P.K, CU_TENSOR_MAP_SWIZZLE_NONE))
+  if (!(kA8 ? make_map_i8(&tmA, Xq, P.M, P.K) : make_map(&tmA, Xq, P.M, P.K, CU_TENSOR_MAP_SWIZZLE_64B)) ||
+      !make_map(&tmB, Wq, P.N, P.K, CU_TENSOR_MAP_SWIZZLE_NONE))
     return FPT_ERR_CUDA;
   if (P.Mq) { if (!make_codes_map(&tmY, P.Mq, P.M, P.N / 4)) return FPT_ERR_CUDA; }
   else if (P.Y) { if (!make_out_map(&tmY, P.Y, P.M, P.swiglu_bf16 ? P.N / 2 : P.N)) return FPT_ERR_CUDA; }
@@ -523,6 +560,7 @@ static int launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, GemmPar
 }  // namespace pair
 
 int gemm_pair_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, const GemmParams& P) {
+  if (P.a_bits == 8) return pair::launch<4, 3, 0, true>(st, Xq, Wq, P);      // Xq: int8 [M, K]
   if (P.Mq) return pair::launch<4, 5, 1>(st, Xq, Wq, P);
   if (P.swiglu_bf16) return pair::launch<4, 5, 2>(st, Xq, Wq, P);
   return pair::launch<4, 5, 0>(st, Xq, Wq, P);

@@ -59,9 +59,23 @@ def test_argument_errors_are_reported_before_any_launch(B):
     assert r == B.ERR_ALIGNMENT
     r = L.fpt_act_quant(None, fake, 4, 128, 128, ctypes.byref(qp), B.SCALE_INPUT, 1e-5, None, None, fake, None)
     assert r == B.ERR_BAD_ARG                          # SCALE_INPUT without s_in
-    q8 = B.QParams(8, True, 0.5, 0)
-    r = L.fpt_act_quant(None, fake, 4, 128, 128, ctypes.byref(q8), B.RMSNORM, 1e-5, None, None, fake, None)
+    q6 = B.QParams(6, True, 0.5, 0)
+    r = L.fpt_act_quant(None, fake, 4, 128, 128, ctypes.byref(q6), B.RMSNORM, 1e-5, None, None, fake, None)
     assert r == B.ERR_UNSUPPORTED
+    q8a = B.QParams(8, False, 0.5, 3)                  # 8-bit codes exist on the symmetric grid only
+    r = L.fpt_act_quant(None, fake, 4, 128, 128, ctypes.byref(q8a), B.RMSNORM, 1e-5, None, None, fake, None)
+    assert r == B.ERR_UNSUPPORTED
+    r = L.fpt_act_quant_dynamic(None, fake, 4, 128, 128, 5, B.RMSNORM, 1e-5, None, fake, None, fake)
+    assert r == B.ERR_UNSUPPORTED
+    r = L.fpt_act_quant_dynamic(None, fake, 4, 128, 128, 4, B.RMSNORM, 1e-5, None, fake, None, None)
+    assert r == B.ERR_BAD_ARG                          # the per-token scales must go somewhere
+    a8 = lambda M, N, K, ws, wsb: (None, fake, fake, M, N, K, fake, B.DTYPE_F32, 0.5, None, None, None, fake, None, ws, wsb)
+    assert L.fpt_w4a8_gemm(*a8(4, 64, 32768, fake, 1 << 30)) == B.ERR_UNSUPPORTED      # (float)acc would round
+    assert L.fpt_w4a8_gemm(*a8(4, 64, 100, fake, 1 << 30)) == B.ERR_UNSUPPORTED
+    assert L.fpt_w4a8_gemm(*a8(4, 64, 128, None, 0)) == B.ERR_WORKSPACE
+    assert L.fpt_w4a8_gemm(*a8(4, 64, 128, fake, 16)) == B.ERR_WORKSPACE
+    assert L.fpt_workspace_bytes(B.OP_GEMM_A8, 300, 512, 1024) == L.fpt_workspace_bytes(B.OP_GEMM, 300, 512, 1024)
+    assert L.fpt_workspace_bytes(B.OP_GEMM_A8, 64, 512, 1024) > L.fpt_workspace_bytes(B.OP_GEMM, 64, 512, 1024)
     qbad = B.QParams(4, False, 0.5, 16)
     r = L.fpt_act_quant(None, fake, 4, 128, 128, ctypes.byref(qbad), B.RMSNORM, 1e-5, None, None, fake, None)
     assert r == B.ERR_BAD_ARG

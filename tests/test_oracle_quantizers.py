@@ -338,3 +338,35 @@ def test_dynamic_quantiser_equivariance_and_degenerate_rows(bits):
     assert np.array_equal(d6, np.ones(3, dtype=F32)) and not c6[0].any()
     assert c6[1, 0] == qmax and c6[1, 1] == -qmax - 1 and c6[1, 2] == 3
     assert c6[2, 0] == -qmax - 1 and c6[2, 1] == -2
+
+
+# --------------------------------------------------------------------------- #
+# 8-bit activation grid (the W4A8 setting)
+# --------------------------------------------------------------------------- #
+def test_eight_bit_grid_idempotence_ties_clamp_and_scalar_brute_force():
+    import struct
+
+    def f(v):
+        return struct.unpack("f", struct.pack("f", v))[0]
+
+    for scale in (0.0371, 1.0, 2.0 ** -5):
+        qp = QParams(8, True, scale)
+        assert (qp.qmin, qp.qmax) == (-128, 127)
+        codes = np.arange(-128, 128)
+        got, _, _, _ = Q.act_quant(Q.dequantize(codes, scale).astype(F32)[None, :], qp, rmsnorm=False)
+        assert got.dtype == np.int8 and got[0].tolist() == codes.tolist()
+    u = np.array([0.5, 1.5, 126.5, 127.5, -127.5, -128.5, 1e9, -1e9, np.nan], dtype=F32)
+    assert Q.round_clamp(u, 0, -128, 127).tolist() == [0, 2, 126, 127, -128, -128, 127, -128, -128]
+    rng = np.random.default_rng(41)
+    x = bf16.round_to_bf16(rng.standard_normal((4, 64)).astype(F32) * 3)
+    s_in = np.exp(rng.standard_normal(4)).astype(F32)
+    qp = QParams(8, True, 0.013)
+    codes, s_out, _, _ = Q.act_quant(x, qp, True, True, 1e-5, s_in)
+    inv = f(1.0 / f(0.013))
+    for t in range(4):
+        ss = f(math.fsum(float(v) * float(v) for v in x[t]))
+        p = f(f(1.0 / f(math.sqrt(f(f(ss / 64.0) + f(1e-5))))) * float(s_in[t]))
+        for k in range(64):
+            q = min(max(round(f(f(float(x[t, k]) * p) * inv)), -128), 127)
+            assert q == int(codes[t, k])
+    assert np.abs(codes.astype(np.int32)).max() > 64          # the wide grid is used
