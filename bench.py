@@ -383,6 +383,16 @@ def run_gpu(args):
                 t_ops += ops
             c5[f"{tokens} tokens"] = {"us_per_layer_linears": t_us, "tokens_per_s": tokens / t_us * 1e6, "TOP/s": t_ops / t_us / 1e6}
         other["configs[4] 70B-class layer linears (act_quant + matmul each; SwiGLU unfused)"] = c5
+        # the dynamic per-token grid and 8-bit activation codes on the fused-QKV shape (quantise + matmul)
+        var = {}
+        for name, kind, bits in (("static W4A4", "linear", 4), ("dynamic W4A4", "linear_dynamic", 4),
+                                 ("dynamic W4A8", "linear_dynamic", 8)):
+            runs, ops, _ = MB.make_case(kind, M_TOK, N_QKV, HID, 4, dev, False, bits)
+            us = MB.time_case_graph(runs, 20)
+            del runs
+            torch.cuda.empty_cache()
+            var[name] = {"us": us, "TOP/s": ops / us / 1e6}
+        other["variants on 2048x6144x4096 (quantise + matmul)"] = var
 
     if rank == 0:
         rows = M_TOK

@@ -6,6 +6,9 @@
     python -m paper_2506_04985_b200.microbench linear    --M 64 --N 14336 --K 4096
     python -m paper_2506_04985_b200.microbench hadamard_quant --M 4096 --K 14336
     python -m paper_2506_04985_b200.microbench mlp       --M 4096 --K 4096 --N 14336      (mlp_hadamard: with the online transform)
+    python -m paper_2506_04985_b200.microbench gemm_a8   --M 2048 --N 6144 --K 4096       (int8 activation codes)
+    python -m paper_2506_04985_b200.microbench linear_dynamic --M 2048 --N 6144 --K 4096 --bits 4
+    python -m paper_2506_04985_b200.microbench act_quant_dynamic --M 2048 --K 4096 --bits 4
 
 Operands are random packed codes / random bf16 values made on the device (timing does
 not depend on the values).  `--sets S` rotates S independent operand sets so that every
@@ -31,7 +34,7 @@ def _bf16(rows, cols, dev):
     return torch.randn((rows, cols), dtype=torch.float32, device=dev).to(torch.bfloat16)
 
 
-def make_case(kind, M, N, K, sets, dev, f16_scales=False):
+def make_case(kind, M, N, K, sets, dev, f16_scales=False, bits=4):
     """Returns (list of zero-argument launchers, algorithmic ops, algorithmic bytes)."""
     sdt = torch.float16 if f16_scales else torch.float32
     ssz = 2 if f16_scales else 4
@@ -66,6 +69,31 @@ def make_case(kind, M, N, K, sets, dev, f16_scales=False):
             out = torch.empty((M, K // 2), dtype=torch.uint8, device=dev)
             runs.append(lambda m=m, s=s, out=out: B.fpt_hadamard_quant(m, qp, B.SCALE_INPUT, s_in=s, out=out))
         return runs, 0.0, 2.5 * M * K + 4.0 * M
+    if kind == "gemm_a8":
+        ws = B.new_workspace(B.OP_GEMM_A8, M, N, K, dev)
+        for _ in range(sets):
+            xq = torch.randint(-128, 128, (M, K), dtype=torch.int8, device=dev)
+            wq = _codes(N, K // 2, dev)
+            sw = torch.rand((N,), device=dev).to(sdt) * 0.01 + 0.001
+            y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+            runs.append(lambda xq=xq, wq=wq, sw=sw, y=y: B.fpt_w4a8_gemm(xq, wq, sw, 0.45, ws=ws, Y=y))
+        return runs, 2.0 * M * N * K, M * K + N * K / 2 + N * ssz + 2.0 * M * N
+    if kind == "act_quant_dynamic":
+        for _ in range(sets):
+            x = _bf16(M, K, dev)
+            out = (torch.empty((M, K // 2), dtype=torch.uint8, device=dev) if bits == 4
+                   else torch.empty((M, K), dtype=torch.int8, device=dev))
+            runs.append(lambda x=x, out=out: B.fpt_act_quant_dynamic(x, bits, B.RMSNORM, 1e-5, want_s_out=False, out=out))
+        return runs, 0.0, (2.0 + bits / 8.0) * M * K + 8.0 * M
+    if kind == "linear_dynamic":
+        for _ in range(sets):
+            x, wq = _bf16(M, K, dev), _codes(N, K // 2, dev)
+            sw = torch.rand((N,), device=dev).to(sdt) * 0.01 + 0.001
+            y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+            ws = B.new_workspace(B.OP_LINEAR_A8 if bits == 8 else B.OP_LINEAR, M, N, K, dev)
+            runs.append(lambda x=x, wq=wq, sw=sw, y=y, ws=ws: B.fpt_w4a4_linear_dynamic(
+                x, wq, sw, bits, B.RMSNORM, 1e-5, want_s_out=False, ws=ws, Y=y))
+        return runs, 2.0 * M * N * K, 2.0 * M * K + N * K / 2 + N * ssz + 2.0 * M * N
     if kind == "linear":
         for _ in range(sets):
             x, wq = _bf16(M, K, dev), _codes(N, K // 2, dev)
@@ -126,7 +154,8 @@ def time_case_graph(runs, reps, warmup=3, replays=5):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("kind", choices=["gemm", "act_quant", "silu_quant", "hadamard_quant", "linear", "mlp", "mlp_hadamard"])
+    ap.add_argument("kind", choices=["gemm", "act_quant", "silu_quant", "hadamard_quant", "linear", "mlp", "mlp_hadamard",
+                                     "gemm_a8", "act_quant_dynamic", "linear_dynamic"])
     ap.add_argument("--M", type=int, default=2048)
     ap.add_argument("--N", type=int, default=4096)
     ap.add_argument("--K", type=int, default=4096)
@@ -134,12 +163,13 @@ def main():
     ap.add_argument("--reps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--f16-scales", action="store_true")
+    ap.add_argument("--bits", type=int, default=4, help="activation bits of the dynamic kinds")
     ap.add_argument("--graph", action="store_true", help="replay the launches from a CUDA graph")
     a = ap.parse_args()
     B.lib()
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
-    runs, ops, nbytes = make_case(a.kind, a.M, a.N, a.K, a.sets, dev, a.f16_scales)
+    runs, ops, nbytes = make_case(a.kind, a.M, a.N, a.K, a.sets, dev, a.f16_scales, a.bits)
     us = time_case_graph(runs, a.reps, a.warmup) if a.graph else time_case(runs, a.reps, a.warmup)
     print(json.dumps({"kind": a.kind, "M": a.M, "N": a.N, "K": a.K, "sets": a.sets, "reps": a.reps,
                       "us": us, "tops": ops / us / 1e6, "gbs": nbytes / us / 1e3}))
