@@ -61,6 +61,15 @@ def test_gemm_post_residual_and_fp16_scales(M, N, K):
     _run(M, N, K, residual=True, f16=True)
 
 
+@pytest.mark.parametrize("M,N,K", [(256, 15392, 128), (256, 16576, 128), (256, 17760, 128), (300, 17768, 256),
+                                   (200, 6152, 128), (513, 248, 256), (2048, 6144, 128)])
+@pytest.mark.parametrize("extras", [False, True])
+def test_gemm_wide_outputs_ragged_column_tiles(M, N, K, extras):
+    """Wide outputs whose width is not a multiple of the 256-column tile (ragged last column tile, more
+    column tiles than CTA pairs), with and without post scale, residual and the asymmetric grid."""
+    _run(M, N, K, seed=5, post=extras, residual=extras, symmetric=not extras, z=9 if extras else 0)
+
+
 def test_gemm_extreme_codes_reach_the_accumulator_bound():
     M, N, K = 130, 264, 28672
     qa = np.full((M, K), -8, dtype=np.int8)
