@@ -110,6 +110,8 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  // quarters of the weight tile the weight converters widen; the activation converters take the rest
+  constexpr int kBShare = kA8 ? 4 : 3;
   const uint32_t rank = cluster_ctarank();             // 0 = leader
   const int pair_id = blockIdx.x >> 1;
   const int num_pairs = gridDim.x >> 1;
@@ -207,6 +209,7 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
       for (int kb = 0; kb < P.kblocks; ++kb) {
         if (!mbar_wait(pk_full(ps), pph, abort_flag, P.status, 5)) { ok = false; break; }
         uint32_t v[32];
+        uint4 cb = make_uint4(0, 0, 0, 0);
         if constexpr (kA8) {
           // int8 codes, 128-byte rows under the 128-byte swizzle.  The weight side orders the 32 codes
           // of a group as 16 even-k then 16 odd-k bytes (that is how the nibbles fall apart); the
@@ -228,12 +231,25 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
           uint4 c[4];
 #pragma unroll
           for (int j = 0; j < 4; ++j) c[j] = *reinterpret_cast<const uint4*>(src + (((uint32_t)j ^ swz) << 4));
+          cb = reinterpret_cast<const uint4*>(smem + L::kPkBOff + ps * L::kPkOp)[kBShare * 128 + r];
 #pragma unroll
           for (int j = 0; j < 4; ++j) widen(c[j], v + 8 * j);
         }
         if (!mbar_wait(op_empty(s), ph ^ 1u, abort_flag, P.status, 6)) { ok = false; break; }
         tc_fence_after();
         tmem_st_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + kAccCols + s * kAStageCols, v);
+        if constexpr (!kA8) {
+          // While the tensor-memory store completes: this warp's share of the WEIGHT tile (its last 32
+          // rows).  The weight converters are the busiest role (measured: 74 % of the k-block period
+          // against 48 % here), so a quarter of their tile is widened by these warps instead.
+          const int id = kBShare * 128 + r;              // 16-byte packed chunk: row id/4, chunk id%4
+          const int br = id >> 2, ch = id & 3;
+          uint32_t w[8];
+          widen(cb, w);
+          uint8_t* rowp = smem + L::kB8Off + s * L::kB8Stage + br * I8_ROW;
+          *reinterpret_cast<uint4*>(rowp + (((2 * ch) ^ (br & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(rowp + (((2 * ch + 1) ^ (br & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+        }
         tmem_wait_st();
         tc_fence_before();
         // The packed tile goes back to TMA only here: its reads have been consumed (the store above
@@ -258,13 +274,13 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
       for (int kb = 0; kb < P.kblocks; ++kb) {
         if (!mbar_wait(pk_full(ps), pph, abort_flag, P.status, 7)) { ok = false; break; }
         const uint4* src = reinterpret_cast<const uint4*>(smem + L::kPkBOff + ps * L::kPkOp);
-        uint4 c[4];
+        uint4 c[kBShare];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) c[i] = src[i * 128 + ctid];
+        for (int i = 0; i < kBShare; ++i) c[i] = src[i * 128 + ctid];
         if (!mbar_wait(op_empty(s), ph ^ 1u, abort_flag, P.status, 8)) { ok = false; break; }
         uint8_t* dst = smem + L::kB8Off + s * L::kB8Stage;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < kBShare; ++i) {
           const int id = i * 128 + ctid;                 // 16-byte packed chunk: row id/4, chunk id%4
           const int r = id >> 2, ch = id & 3;
           uint32_t w[8];
