@@ -85,7 +85,10 @@ gemm_w4a4_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
   using L = Smem;
   const GemmParams& P = D.g;
   extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  // aligned to 1024 bytes by an offset on the shared-memory array itself (a round trip through an
+  // integer would leave a generic pointer: generic loads and stores, and no way for the compiler to
+  // tell shared from global accesses apart)
+  uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   const uint32_t sbase = smem_u32(smem);
   const uint32_t bar0 = sbase + L::kBarOff;
   auto pk_full = [&](int s) { return bar0 + 8u * s; };
