@@ -86,10 +86,11 @@ __device__ __forceinline__ void load_scales8(const void* sw, int scale_dtype, in
 
 // kFuse: 0 plain scale-factor epilogue; 1 SwiGLU product + quantiser (codes out); 2 SwiGLU product
 // (bf16 out).  Separate instantiations keep the plain epilogue's register budget free of the others.
-template <int NS, int NPK, int kFuse, bool kA8 = false>
+template <int NS, int NPK, int kFuse, bool kA8 = false, int kTN = TN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                      const __grid_constant__ CUtensorMap tmY, const GemmParams P) {
+                      const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmYt,
+                      const GemmParams P) {
   using L = Smem<NS, NPK, kA8>;
   static_assert(!kA8 || kFuse == 0, "8-bit activations: plain epilogue only");
   extern __shared__ uint8_t smem_raw[];
@@ -118,6 +119,12 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
   const uint32_t rank = cluster_ctarank();             // 0 = leader
   const int pair_id = blockIdx.x >> 1;
   const int num_pairs = gridDim.x >> 1;
+  // Width of the output tile.  The plain epilogue also exists for 208, 224 and 240 columns: the host
+  // picks the width that wastes the least of the last round of tiles (the kernel is bound by the
+  // tensor pipe, so a narrower tile takes proportionally less time).  The fused epilogues need 256.
+  static_assert(kTN == TN || (kFuse == 0 && kTN >= 208 && kTN % 16 == 0), "tile width");
+  constexpr int tn = kTN;
+  constexpr int hb = tn >> 1;                          // weight rows of the tile this CTA holds
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < NPK; ++s) { mbar_init(pk_full(s), 1); mbar_init(pk_empty(s), 8); }
@@ -129,7 +136,7 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     fence_mbar_init();
     prefetch_tmap(&tmA);
     prefetch_tmap(&tmB);
-    if (P.Y || kFuse == 1) prefetch_tmap(&tmY);
+    if (P.Y || kFuse == 1) { prefetch_tmap(&tmY); if (tn < TN) prefetch_tmap(&tmYt); }
   }
   if (warp == 1) {
     tmem_alloc_pair(sbase + L::kMiscOff, kTmemCols);
@@ -155,10 +162,10 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
       bool ok = true;
       for (int tile = pair_id; ok && tile < P.num_tiles; tile += num_pairs) {
         const int m0 = (tile % P.tiles_m) * TM + (int)rank * HR;
-        const int n0 = (tile / P.tiles_m) * TN + (int)rank * HR;
+        const int n0 = (tile / P.tiles_m) * tn + (int)rank * hb;
         for (int kb = 0; kb < P.kblocks; ++kb) {
           if (!mbar_wait(pk_empty(s), ph ^ 1u, abort_flag, P.status, 1)) { ok = false; break; }
-          mbar_arrive_expect_tx(pk_full(s), L::kPkOpA + L::kPkOp);
+          mbar_arrive_expect_tx(pk_full(s), L::kPkOpA + (uint32_t)hb * PK_ROW);
           tma_load_2d(sbase + L::kPkAOff + s * L::kPkOpA, &tmA, pk_full(s), kb * (kA8 ? I8_ROW : PK_ROW), m0);
           tma_load_2d(sbase + L::kPkBOff + s * L::kPkOp, &tmB, pk_full(s), kb * PK_ROW, n0);
           armed |= 1u << s;
@@ -177,7 +184,7 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA only)
     if (rank == 0 && lane == 0) {
-      const uint32_t idesc = umma_idesc_i8(TM, TN, !P.a_unsigned, true);
+      const uint32_t idesc = umma_idesc_i8(TM, tn, !P.a_unsigned, true);
       int s = 0; uint32_t ph = 0; int it = 0;
       for (int tile = pair_id; tile < P.num_tiles; tile += num_pairs, ++it) {
         if (!mbar_wait_cluster(acc_empty, (it & 1) ^ 1u, abort_flag, P.status, 2)) break;
@@ -247,11 +254,13 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
           // against 48 % here), so a quarter of their tile is widened by these warps instead.
           const int id = kBShare * 128 + r;              // 16-byte packed chunk: row id/4, chunk id%4
           const int br = id >> 2, ch = id & 3;
-          uint32_t w[8];
-          widen(cb, w);
-          uint8_t* rowp = smem + L::kB8Off + s * L::kB8Stage + br * I8_ROW;
-          *reinterpret_cast<uint4*>(rowp + (((2 * ch) ^ (br & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-          *reinterpret_cast<uint4*>(rowp + (((2 * ch + 1) ^ (br & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+          if (br < hb) {                                 // a narrower tile has fewer weight rows
+            uint32_t w[8];
+            widen(cb, w);
+            uint8_t* rowp = smem + L::kB8Off + s * L::kB8Stage + br * I8_ROW;
+            *reinterpret_cast<uint4*>(rowp + (((2 * ch) ^ (br & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+            *reinterpret_cast<uint4*>(rowp + (((2 * ch + 1) ^ (br & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+          }
         }
         tmem_wait_st();
         tc_fence_before();
@@ -286,6 +295,7 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         for (int i = 0; i < kBShare; ++i) {
           const int id = i * 128 + ctid;                 // 16-byte packed chunk: row id/4, chunk id%4
           const int r = id >> 2, ch = id & 3;
+          if (i == 3 && r >= hb) continue;               // (int8 activations: this role has all four quarters)
           uint32_t w[8];
           widen(c[i], w);
           uint8_t* rowp = dst + r * I8_ROW;
@@ -319,12 +329,13 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     for (int tile = pair_id; tile < P.num_tiles; tile += num_pairs, ++it) {
       const int b = it & 1; const uint32_t bph = (it >> 1) & 1;
       const int m0 = (tile % P.tiles_m) * TM + (int)rank * HR;
-      const int nt = (tile / P.tiles_m) * TN;            // first column of the tile
+      const int nt = (tile / P.tiles_m) * tn;            // first column of the tile
+      const int n_end = nt + tn < P.N ? nt + tn : P.N;   // one past the tile's last valid column
       // scale factors of the tile's columns -> shared memory, while the matmul of the tile runs
       {
         const int n = nt + etid;
-        sw_s[b * TN + etid] = n < P.N ? load_scale(P.sw, P.scale_dtype, n) : 0.0f;
-        zw_s[b * TN + etid] = (P.wsum && n < P.N) ? P.zero_point * __ldg(P.wsum + n) : 0;
+        sw_s[b * TN + etid] = n < n_end ? load_scale(P.sw, P.scale_dtype, n) : 0.0f;
+        zw_s[b * TN + etid] = (P.wsum && n < n_end) ? P.zero_point * __ldg(P.wsum + n) : 0;
       }
       const int row = m0 + r;
       const bool row_ok = row < P.M;
@@ -394,7 +405,7 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
           int a[8];
 #pragma unroll
           for (int j = 0; j < 8; ++j) a[j] = (((int)v[ch * 32 + g * 8 + j]) >> kShift) - zws[ch * 32 + g * 8 + j];
-          if (P.acc_out && row_ok && col < P.N) {
+          if (P.acc_out && row_ok && col < n_end) {
             int4* o = reinterpret_cast<int4*>(P.acc_out + rowoff + col);
             o[0] = make_int4(a[0], a[1], a[2], a[3]);
             o[1] = make_int4(a[4], a[5], a[6], a[7]);
@@ -407,7 +418,7 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
               const float af = magic_ok ? __fsub_rn(__int_as_float(0x4B400000 + a[j]), 12582912.0f) : (float)a[j];
               y[j] = __fmul_rn(__fmul_rn(af, sws[ch * 32 + g * 8 + j]), c);
             }
-            if (P.residual && row_ok && col < P.N) {
+            if (P.residual && row_ok && col < n_end) {
               const uint4 r4 = __ldg(reinterpret_cast<const uint4*>(P.residual + rowoff + col));
               const uint32_t rw[4] = {r4.x, r4.y, r4.z, r4.w};
 #pragma unroll
@@ -422,7 +433,14 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             o.z = f32_to_bf16_bits(y[4]) | (f32_to_bf16_bits(y[5]) << 16);
             o.w = f32_to_bf16_bits(y[6]) | (f32_to_bf16_bits(y[7]) << 16);
             const int chunk = (ch & 1) * 4 + g;          // 16-byte chunk of the slab row; 128-byte swizzle
-            *reinterpret_cast<uint4*>(slab + ((chunk ^ (r & 7)) << 4)) = o;
+            if (tn < TN && half == 1 && ch >= 2) {
+              // last slab of a narrower tile: tn - 192 columns, dense rows, no swizzle (its own tensor map)
+              constexpr int tail_bytes = (tn - 192) * 2;
+              if (chunk * 16 < tail_bytes)
+                *reinterpret_cast<uint4*>(smem + L::kStgOff + 3 * L::kStgSlab + r * tail_bytes + chunk * 16) = o;
+            } else {
+              *reinterpret_cast<uint4*>(slab + ((chunk ^ (r & 7)) << 4)) = o;
+            }
           }
         }
       }
@@ -440,7 +458,7 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             tma_store_2d(&tmY, s0, nt / 2 + half * 64, m0);            // 128 rows x 64 products
           } else {
             tma_store_2d(&tmY, s0, nt + half * 128, m0);
-            tma_store_2d(&tmY, s0 + L::kStgSlab, nt + half * 128 + 64, m0);
+            tma_store_2d((tn < TN && half == 1) ? &tmYt : &tmY, s0 + L::kStgSlab, nt + half * 128 + 64, m0);
           }
           tma_store_commit();
           tma_store_wait_read();
@@ -484,12 +502,12 @@ static EncodeTiledFn encode_fn() {
 }
 
 // Tensor map over a packed [rows, K/2]-byte matrix; one box = 128 rows of one k-block (64 bytes each).
-static bool make_map(CUtensorMap* m, const void* base, int rows, int K, CUtensorMapSwizzle swz) {
+static bool make_map(CUtensorMap* m, const void* base, int rows, int K, CUtensorMapSwizzle swz, int box_rows = HR) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   const cuuint64_t dims[2] = {(cuuint64_t)(K / 2), (cuuint64_t)rows};
   const cuuint64_t strides[1] = {(cuuint64_t)(K / 2)};
-  const cuuint32_t box[2] = {(cuuint32_t)PK_ROW, (cuuint32_t)HR};
+  const cuuint32_t box[2] = {(cuuint32_t)PK_ROW, (cuuint32_t)box_rows};
   const cuuint32_t estr[2] = {1, 1};
   return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -510,16 +528,32 @@ static bool make_map_i8(CUtensorMap* m, const void* base, int rows, int K) {
 }
 
 // Tensor map over the bf16 output [M, N]; one box = 128 rows x 64 columns, 128-byte swizzle in shared memory.
-static bool make_out_map(CUtensorMap* m, const void* base, int M, int N) {
+// (box_cols < 64: the narrow last slab of a tile that is less than 256 columns wide; dense rows, no swizzle.)
+static bool make_out_map(CUtensorMap* m, const void* base, int M, int N, int box_cols = 64) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   const cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
   const cuuint64_t strides[1] = {(cuuint64_t)N * 2};
-  const cuuint32_t box[2] = {64, (cuuint32_t)HR};
+  const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)HR};
   const cuuint32_t estr[2] = {1, 1};
   return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+            CU_TENSOR_MAP_INTERLEAVE_NONE, box_cols == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+            CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Tile width for the plain epilogue: tiles are dealt out in rounds of `pairs`, a tile's time is
+// proportional to its width (tensor-pipe bound), so the width with the smallest rounds x width wins;
+// among equal costs the widest (fewest tiles, least activation traffic).
+static int choose_tn(int M, int N, int pairs) {
+  const int tiles_m = (M + TM - 1) / TM;
+  int best = TN;
+  long long best_cost = -1;
+  for (int tn = TN; tn >= 208; tn -= 16) {
+    const long long tiles = (long long)tiles_m * ((N + tn - 1) / tn);
+    const long long cost = ((tiles + pairs - 1) / pairs) * tn;
+    if (best_cost < 0 || cost * 100 < best_cost * 98) { best_cost = cost; best = tn; }
+  }
+  return best;
 }
 
 // Tensor map over the packed codes [M, N/4 bytes] the fused SwiGLU epilogue writes; one box = 128 rows x 32 bytes.
@@ -535,10 +569,10 @@ static bool make_codes_map(CUtensorMap* m, const void* base, int M, int row_byte
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int NS, int NPK, int kFuse, bool kA8 = false>
+template <int NS, int NPK, int kFuse, bool kA8 = false, int kTN = TN>
 static int launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, GemmParams P) {
   using L = Smem<NS, NPK, kA8>;
-  auto kern = gemm_w4a4_pair_kernel<NS, NPK, kFuse, kA8>;
+  auto kern = gemm_w4a4_pair_kernel<NS, NPK, kFuse, kA8, kTN>;
   static int max_pairs = 0;                 // co-resident CTA pairs on this device
   if (!max_pairs) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kAlloc) != cudaSuccess)
@@ -561,28 +595,54 @@ static int launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, GemmPar
     }
     max_pairs = n > 0 ? n : 1;
   }
-  CUtensorMap tmA, tmB, tmY;
+  CUtensorMap tmA, tmB, tmY, tmYt;
   if (!(kA8 ? make_map_i8(&tmA, Xq, P.M, P.K) : make_map(&tmA, Xq, P.M, P.K, CU_TENSOR_MAP_SWIZZLE_64B)) ||
-      !make_map(&tmB, Wq, P.N, P.K, CU_TENSOR_MAP_SWIZZLE_NONE))
+      !make_map(&tmB, Wq, P.N, P.K, CU_TENSOR_MAP_SWIZZLE_NONE, kTN / 2))
     return FPT_ERR_CUDA;
   if (P.Mq) { if (!make_codes_map(&tmY, P.Mq, P.M, P.N / 4)) return FPT_ERR_CUDA; }
   else if (P.Y) { if (!make_out_map(&tmY, P.Y, P.M, P.swiglu_bf16 ? P.N / 2 : P.N)) return FPT_ERR_CUDA; }
   else tmY = tmA;                                                                  // unused without an output tile
+  tmYt = tmY;
+  if (kTN < TN && P.Y && !make_out_map(&tmYt, P.Y, P.M, P.N, kTN - 192)) return FPT_ERR_CUDA;
   P.tiles_m = (P.M + TM - 1) / TM;
-  P.num_tiles = P.tiles_m * ((P.N + TN - 1) / TN);
+  P.num_tiles = P.tiles_m * ((P.N + kTN - 1) / kTN);
   P.kblocks = P.K / BK;
   const int pairs = P.num_tiles < max_pairs ? P.num_tiles : max_pairs;
-  kern<<<2 * pairs, kThreads, L::kAlloc, st>>>(tmA, tmB, tmY, P);
+  kern<<<2 * pairs, kThreads, L::kAlloc, st>>>(tmA, tmB, tmY, tmYt, P);
   return cudaGetLastError() == cudaSuccess ? FPT_OK : FPT_ERR_CUDA;
 }
 
 }  // namespace pair
 
+static int device_pairs() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0, sms = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    n = sms >= 2 ? sms / 2 : 1;
+  }
+  return n;
+}
+
 int gemm_pair_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, const GemmParams& P) {
-  if (P.a_bits == 8) return pair::launch<4, 3, 0, true>(st, Xq, Wq, P);      // Xq: int8 [M, K]
   if (P.Mq) return pair::launch<4, 5, 1>(st, Xq, Wq, P);
   if (P.swiglu_bf16) return pair::launch<4, 5, 2>(st, Xq, Wq, P);
-  return pair::launch<4, 5, 0>(st, Xq, Wq, P);
+  const int tn = pair::choose_tn(P.M, P.N, device_pairs());
+  if (P.a_bits == 8) {                                                        // Xq: int8 [M, K]
+    switch (tn) {
+      case 240: return pair::launch<4, 3, 0, true, 240>(st, Xq, Wq, P);
+      case 224: return pair::launch<4, 3, 0, true, 224>(st, Xq, Wq, P);
+      case 208: return pair::launch<4, 3, 0, true, 208>(st, Xq, Wq, P);
+      default:  return pair::launch<4, 3, 0, true, 256>(st, Xq, Wq, P);
+    }
+  }
+  switch (tn) {
+    case 240: return pair::launch<4, 5, 0, false, 240>(st, Xq, Wq, P);
+    case 224: return pair::launch<4, 5, 0, false, 224>(st, Xq, Wq, P);
+    case 208: return pair::launch<4, 5, 0, false, 208>(st, Xq, Wq, P);
+    default:  return pair::launch<4, 5, 0, false, 256>(st, Xq, Wq, P);
+  }
 }
 
 }  // namespace fpt
