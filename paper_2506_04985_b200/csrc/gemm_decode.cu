@@ -339,16 +339,21 @@ gemm_w4a4_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         }
       }
       if (finalize && n_ok) {
+        // (everything the loop needs from the parameter block is read once, here)
+        const int m_tok = P.M;
+        const size_t ldy = (size_t)P.N;
+        int32_t* const acc_out = P.acc_out ? P.acc_out + n : nullptr;
+        __nv_bfloat16* const yp = P.Y ? P.Y + n : nullptr;
+        const __nv_bfloat16* const resp = P.residual ? P.residual + n : nullptr;
 #pragma unroll
         for (int t = 0; t < kMaxTok; ++t) {
-          if (t < P.M) {
+          if (t < m_tok) {
             const int a = (((int)v[t]) >> 8) - zw;
-            if (P.acc_out) P.acc_out[(size_t)t * P.N + n] = a;
-            if (P.Y) {
+            if (acc_out) acc_out[(size_t)t * ldy] = a;
+            if (yp) {
               float y = __fmul_rn(__fmul_rn((float)a, swn), c_s[t]);
-              if (P.residual)
-                y = __fadd_rn(y, __fmul_rn(__bfloat162float(P.residual[(size_t)t * P.N + n]), rs_s[t]));
-              P.Y[(size_t)t * P.N + n] = __float2bfloat16_rn(y);
+              if (resp) y = __fadd_rn(y, __fmul_rn(__bfloat162float(resp[(size_t)t * ldy]), rs_s[t]));
+              yp[(size_t)t * ldy] = __float2bfloat16_rn(y);
             }
           }
         }
