@@ -112,6 +112,13 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
   volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(smem + L::kMiscOff);
   volatile uint32_t* abort_flag = misc + 1;
 
+  // the parameter block is read once, here (not inside the role loops)
+  uint32_t* const status_w = P.status;
+  const int kblocks = P.kblocks, num_tiles = P.num_tiles, tiles_m = P.tiles_m;
+  const int n_cols = P.N, m_rows = P.M;
+  int32_t* const acc_out_p = P.acc_out;
+  const __nv_bfloat16* const residual_p = P.residual;
+  __nv_bfloat16* const y_out_p = P.Y;
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   // quarters of the weight tile the weight converters widen; the activation converters take the rest
@@ -136,7 +143,7 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     fence_mbar_init();
     prefetch_tmap(&tmA);
     prefetch_tmap(&tmB);
-    if (P.Y || kFuse == 1) { prefetch_tmap(&tmY); if (tn < TN) prefetch_tmap(&tmYt); }
+    if (y_out_p || kFuse == 1) { prefetch_tmap(&tmY); if (tn < TN) prefetch_tmap(&tmYt); }
   }
   if (warp == 1) {
     tmem_alloc_pair(sbase + L::kMiscOff, kTmemCols);
@@ -160,11 +167,11 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
       int s = 0; uint32_t ph = 0;
       uint32_t armed = 0, armed_par = 0;
       bool ok = true;
-      for (int tile = pair_id; ok && tile < P.num_tiles; tile += num_pairs) {
-        const int m0 = (tile % P.tiles_m) * TM + (int)rank * HR;
-        const int n0 = (tile / P.tiles_m) * tn + (int)rank * hb;
-        for (int kb = 0; kb < P.kblocks; ++kb) {
-          if (!mbar_wait(pk_empty(s), ph ^ 1u, abort_flag, P.status, 1)) { ok = false; break; }
+      for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs) {
+        const int m0 = (tile % tiles_m) * TM + (int)rank * HR;
+        const int n0 = (tile / tiles_m) * tn + (int)rank * hb;
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!mbar_wait(pk_empty(s), ph ^ 1u, abort_flag, status_w, 1)) { ok = false; break; }
           mbar_arrive_expect_tx(pk_full(s), L::kPkOpA + (uint32_t)hb * PK_ROW);
           tma_load_2d(sbase + L::kPkAOff + s * L::kPkOpA, &tmA, pk_full(s), kb * (kA8 ? I8_ROW : PK_ROW), m0);
           tma_load_2d(sbase + L::kPkBOff + s * L::kPkOp, &tmB, pk_full(s), kb * PK_ROW, n0);
@@ -186,12 +193,12 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     if (rank == 0 && lane == 0) {
       const uint32_t idesc = umma_idesc_i8(TM, tn, !P.a_unsigned, true);
       int s = 0; uint32_t ph = 0; int it = 0;
-      for (int tile = pair_id; tile < P.num_tiles; tile += num_pairs, ++it) {
-        if (!mbar_wait_cluster(acc_empty, (it & 1) ^ 1u, abort_flag, P.status, 2)) break;
+      for (int tile = pair_id; tile < num_tiles; tile += num_pairs, ++it) {
+        if (!mbar_wait_cluster(acc_empty, (it & 1) ^ 1u, abort_flag, status_w, 2)) break;
         tc_fence_after();
         bool ok = true;
-        for (int kb = 0; kb < P.kblocks; ++kb) {
-          if (!mbar_wait_cluster(op_full(s), ph, abort_flag, P.status, 3)) { ok = false; break; }
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!mbar_wait_cluster(op_full(s), ph, abort_flag, status_w, 3)) { ok = false; break; }
           tc_fence_after();
           const uint64_t bdesc = umma_desc_kmajor_sw128(sbase + L::kB8Off + s * L::kB8Stage);
           const uint32_t a_tmem = tmem_base + kAccCols + s * kAStageCols;
@@ -215,9 +222,9 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     const uint32_t op_full_leader = map_to_cta(op_full(0), 0);
     int ps = 0, s = 0; uint32_t pph = 0, ph = 0;
     bool ok = true;
-    for (int tile = pair_id; ok && tile < P.num_tiles; tile += num_pairs) {
-      for (int kb = 0; kb < P.kblocks; ++kb) {
-        if (!mbar_wait(pk_full(ps), pph, abort_flag, P.status, 5)) { ok = false; break; }
+    for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs) {
+      for (int kb = 0; kb < kblocks; ++kb) {
+        if (!mbar_wait(pk_full(ps), pph, abort_flag, status_w, 5)) { ok = false; break; }
         uint32_t v[32];
         uint4 cb = make_uint4(0, 0, 0, 0);
         if constexpr (kA8) {
@@ -245,7 +252,7 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
 #pragma unroll
           for (int j = 0; j < 4; ++j) widen(c[j], v + 8 * j);
         }
-        if (!mbar_wait(op_empty(s), ph ^ 1u, abort_flag, P.status, 6)) { ok = false; break; }
+        if (!mbar_wait(op_empty(s), ph ^ 1u, abort_flag, status_w, 6)) { ok = false; break; }
         tc_fence_after();
         tmem_st_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + kAccCols + s * kAStageCols, v);
         if constexpr (!kA8) {
@@ -282,14 +289,14 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     const uint32_t op_full_leader = map_to_cta(op_full(0), 0);
     int ps = 0, s = 0; uint32_t pph = 0, ph = 0;
     bool ok = true;
-    for (int tile = pair_id; ok && tile < P.num_tiles; tile += num_pairs) {
-      for (int kb = 0; kb < P.kblocks; ++kb) {
-        if (!mbar_wait(pk_full(ps), pph, abort_flag, P.status, 7)) { ok = false; break; }
+    for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs) {
+      for (int kb = 0; kb < kblocks; ++kb) {
+        if (!mbar_wait(pk_full(ps), pph, abort_flag, status_w, 7)) { ok = false; break; }
         const uint4* src = reinterpret_cast<const uint4*>(smem + L::kPkBOff + ps * L::kPkOp);
         uint4 c[kBShare];
 #pragma unroll
         for (int i = 0; i < kBShare; ++i) c[i] = src[i * 128 + ctid];
-        if (!mbar_wait(op_empty(s), ph ^ 1u, abort_flag, P.status, 8)) { ok = false; break; }
+        if (!mbar_wait(op_empty(s), ph ^ 1u, abort_flag, status_w, 8)) { ok = false; break; }
         uint8_t* dst = smem + L::kB8Off + s * L::kB8Stage;
 #pragma unroll
         for (int i = 0; i < kBShare; ++i) {
@@ -326,11 +333,11 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     const bool magic_ok = kA8 ? P.K < 4096 : P.K <= 32768;   // |acc| < 2^22: int -> float by exponent trick
     const bool issuer = quad == 0 && lane == 0;          // issues the TMA stores of its half
     int it = 0;
-    for (int tile = pair_id; tile < P.num_tiles; tile += num_pairs, ++it) {
+    for (int tile = pair_id; tile < num_tiles; tile += num_pairs, ++it) {
       const int b = it & 1; const uint32_t bph = (it >> 1) & 1;
-      const int m0 = (tile % P.tiles_m) * TM + (int)rank * HR;
-      const int nt = (tile / P.tiles_m) * tn;            // first column of the tile
-      const int n_end = nt + tn < P.N ? nt + tn : P.N;   // one past the tile's last valid column
+      const int m0 = (tile % tiles_m) * TM + (int)rank * HR;
+      const int nt = (tile / tiles_m) * tn;            // first column of the tile
+      const int n_end = nt + tn < n_cols ? nt + tn : n_cols;   // one past the tile's last valid column
       // scale factors of the tile's columns -> shared memory, while the matmul of the tile runs
       {
         const int n = nt + etid;
@@ -338,20 +345,20 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         zw_s[b * TN + etid] = (P.wsum && n < n_end) ? P.zero_point * __ldg(P.wsum + n) : 0;
       }
       const int row = m0 + r;
-      const bool row_ok = row < P.M;
+      const bool row_ok = row < m_rows;
       float c = P.act_scale, rs = 1.0f;
       if (row_ok && P.post) c = __fmul_rn(P.act_scale, __ldg(P.post + row));
       if (row_ok && P.res_scale) rs = __ldg(P.res_scale + row);
       const float sn = (kFuse == 1 && row_ok) ? __ldg(P.mid_scale + row) : 0.0f;
       __syncwarp();
       if (lane == 0) mbar_arrive(sc_full(b));
-      if (!mbar_wait(sc_full(b), bph, abort_flag, P.status, 9)) break;
+      if (!mbar_wait(sc_full(b), bph, abort_flag, status_w, 9)) break;
       // the staging half must have been read by the TMA store of the previous tile
-      if ((P.Y || kFuse == 1) && !mbar_wait(stg_empty(half), (it & 1) ^ 1u, abort_flag, P.status, 10)) break;
-      if (!mbar_wait(acc_full, it & 1, abort_flag, P.status, 4)) break;
+      if ((y_out_p || kFuse == 1) && !mbar_wait(stg_empty(half), (it & 1) ^ 1u, abort_flag, status_w, 10)) break;
+      if (!mbar_wait(acc_full, it & 1, abort_flag, status_w, 4)) break;
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + half * 128;
-      const size_t rowoff = (size_t)row * (size_t)P.N;
+      const size_t rowoff = (size_t)row * (size_t)n_cols;
       const float* sws = sw_s + b * TN + half * 128;
       const int* zws = zw_s + b * TN + half * 128;
       // all 128 accumulators of this thread's row -> registers, then the accumulator is free again
@@ -405,12 +412,12 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
           int a[8];
 #pragma unroll
           for (int j = 0; j < 8; ++j) a[j] = (((int)v[ch * 32 + g * 8 + j]) >> kShift) - zws[ch * 32 + g * 8 + j];
-          if (P.acc_out && row_ok && col < n_end) {
-            int4* o = reinterpret_cast<int4*>(P.acc_out + rowoff + col);
+          if (acc_out_p && row_ok && col < n_end) {
+            int4* o = reinterpret_cast<int4*>(acc_out_p + rowoff + col);
             o[0] = make_int4(a[0], a[1], a[2], a[3]);
             o[1] = make_int4(a[4], a[5], a[6], a[7]);
           }
-          if (P.Y) {
+          if (y_out_p) {
             float y[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
@@ -418,8 +425,8 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
               const float af = magic_ok ? __fsub_rn(__int_as_float(0x4B400000 + a[j]), 12582912.0f) : (float)a[j];
               y[j] = __fmul_rn(__fmul_rn(af, sws[ch * 32 + g * 8 + j]), c);
             }
-            if (P.residual && row_ok && col < n_end) {
-              const uint4 r4 = __ldg(reinterpret_cast<const uint4*>(P.residual + rowoff + col));
+            if (residual_p && row_ok && col < n_end) {
+              const uint4 r4 = __ldg(reinterpret_cast<const uint4*>(residual_p + rowoff + col));
               const uint32_t rw[4] = {r4.x, r4.y, r4.z, r4.w};
 #pragma unroll
               for (int j = 0; j < 4; ++j) {
@@ -445,12 +452,12 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         }
       }
       }
-      if (P.Y || kFuse == 1) {
+      if (y_out_p || kFuse == 1) {
         fence_proxy_async_smem();                        // staged tile -> visible to the TMA engine
         __syncwarp();
         if (lane == 0) mbar_arrive(stg_full(half));
         if (issuer) {
-          if (!mbar_wait(stg_full(half), it & 1, abort_flag, P.status, 11)) break;
+          if (!mbar_wait(stg_full(half), it & 1, abort_flag, status_w, 11)) break;
           const uint32_t s0 = sbase + L::kStgOff + (half * 2) * L::kStgSlab;
           if constexpr (kFuse == 1) {
             tma_store_2d(&tmY, s0, nt / 4 + half * 32, m0);            // 128 rows x 32 bytes of packed codes
