@@ -337,6 +337,14 @@ int gemm_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, const Gem
   if (P.M <= 16) return gemm_decode_small_launch(st, Xq, Wq, P);
   if (P.M <= 64 && P.scratch) return gemm_decode_launch(st, Xq, Wq, P, P.scratch);
   if (P.M > 128 && P.N > 128) return gemm_pair_launch(st, Xq, Wq, P);
+  if (P.M > 64 && P.N > 128) {
+    // 65..128 tokens: the CTA-pair kernel (half of its 256 activation rows empty) still beats the
+    // one-CTA kernel per k-block (measured 0.5 against 0.68 us), unless it needs more rounds of tiles
+    const int sms = num_sms(), pairs = sms >= 2 ? sms / 2 : 1;
+    const int rounds_1 = ((P.N + 255) / 256 + sms - 1) / sms;
+    const int rounds_2 = ((P.N + 207) / 208 + pairs - 1) / pairs;
+    if (rounds_2 * 3 < rounds_1 * 4) return gemm_pair_launch(st, Xq, Wq, P);
+  }
   if (P.N <= 64) return launch_gemm<64, 4, 4, 8>(st, Xq, Wq, P);
   if (P.N <= 128) return launch_gemm<128, 4, 4, 8>(st, Xq, Wq, P);
   return launch_gemm<256, 3, 3, 8>(st, Xq, Wq, P);
