@@ -57,7 +57,7 @@ struct Smem {
   static constexpr int kStgSlab = HR * 128;                         // 16 KB, 128-byte rows, 128-byte swizzle
   static constexpr int kScaleOff = kStgOff + 4 * kStgSlab;          // 2 x 256 floats (sw) + 2 x 256 ints (z * wsum)
   static constexpr int kBarOff = kScaleOff + 2 * TN * 4 * 2;
-  static constexpr int kNumBars = 2 * NPK + 2 * NS + 2 + 2 + 2 + 2;
+  static constexpr int kNumBars = 2 * NPK + 2 * NS + 2 + 2 + 2 + 2 + 2;
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;           // tmem base, abort flag
   static constexpr int kBytes = kMiscOff + 16;
   static constexpr int kAlloc = kBytes + 1024;                      // slack to align the base to 1024
@@ -90,6 +90,7 @@ template <int NS, int NPK, int kFuse, bool kA8 = false, int kTN = TN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                       const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmYt,
+                      const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmRt,
                       const GemmParams P) {
   using L = Smem<NS, NPK, kA8>;
   static_assert(!kA8 || kFuse == 0, "8-bit activations: plain epilogue only");
@@ -109,6 +110,7 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
   auto sc_full = [&](int b) { return acc_full + 16u + 8u * b; };               // scales of a tile are in shared memory
   auto stg_full = [&](int h) { return acc_full + 32u + 8u * h; };              // a 128-column half of the tile is staged
   auto stg_empty = [&](int h) { return acc_full + 48u + 8u * h; };             // ... and has been read by its TMA store
+  auto res_full = [&](int h) { return acc_full + 64u + 8u * h; };              // the residual of a half has arrived in the staging slabs
   volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(smem + L::kMiscOff);
   volatile uint32_t* abort_flag = misc + 1;
 
@@ -138,7 +140,7 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     for (int s = 0; s < NS; ++s) { mbar_init(op_full(s), 16); mbar_init(op_empty(s), 1); }
     mbar_init(acc_full, 1);
     mbar_init(acc_empty, 2 * kEpiWarps);
-    for (int b = 0; b < 2; ++b) { mbar_init(sc_full(b), kEpiWarps); mbar_init(stg_full(b), 4); mbar_init(stg_empty(b), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(sc_full(b), kEpiWarps); mbar_init(stg_full(b), 4); mbar_init(stg_empty(b), 1); mbar_init(res_full(b), 1); }
     misc[1] = 0;
     fence_mbar_init();
     prefetch_tmap(&tmA);
@@ -331,8 +333,10 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     const int r = quad * 32 + lane;                      // row of the CTA's 128
     constexpr int kShift = kA8 ? 4 : 8;                  // both operands carry a factor 16, int8 activations none
     const bool magic_ok = kA8 ? P.K < 4096 : P.K <= 32768;   // |acc| < 2^22: int -> float by exponent trick
-    const bool issuer = quad == 0 && lane == 0;          // issues the TMA stores of its half
+    const bool issuer = quad == 0 && lane == 0;          // issues the TMA stores (and residual loads) of its half
+    const bool use_res = kFuse == 0 && residual_p != nullptr && y_out_p != nullptr;
     int it = 0;
+    int res_armed = 0, res_seen = 0;                     // residual loads issued / seen to arrive (tiles, 1-based)
     for (int tile = pair_id; tile < num_tiles; tile += num_pairs, ++it) {
       const int b = it & 1; const uint32_t bph = (it >> 1) & 1;
       const int m0 = (tile % tiles_m) * TM + (int)rank * HR;
@@ -355,6 +359,20 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
       if (!mbar_wait(sc_full(b), bph, abort_flag, status_w, 9)) break;
       // the staging half must have been read by the TMA store of the previous tile
       if ((y_out_p || kFuse == 1) && !mbar_wait(stg_empty(half), (it & 1) ^ 1u, abort_flag, status_w, 10)) break;
+      if constexpr (kFuse == 0) {
+        // The residual tile of this half travels by TMA into the staging slabs, in the layout the output
+        // will have there, while the matmul of the tile still runs; each thread later reads the 16 bytes
+        // it is about to overwrite.  (Read straight from global memory, one row per thread, these loads
+        // were uncoalesced and made the epilogue the slow side.)
+        if (use_res && issuer) {
+          const uint32_t s0 = sbase + L::kStgOff + (half * 2) * L::kStgSlab;
+          const uint32_t second = (tn < TN && half == 1) ? (uint32_t)HR * (uint32_t)(tn - 192) * 2u : (uint32_t)L::kStgSlab;
+          mbar_arrive_expect_tx(res_full(half), (uint32_t)L::kStgSlab + second);
+          tma_load_2d(s0, &tmR, res_full(half), nt + half * 128, m0);
+          tma_load_2d(s0 + L::kStgSlab, (tn < TN && half == 1) ? &tmRt : &tmR, res_full(half), nt + half * 128 + 64, m0);
+          res_armed = it + 1;
+        }
+      }
       if (!mbar_wait(acc_full, it & 1, abort_flag, status_w, 4)) break;
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + half * 128;
@@ -403,6 +421,8 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
           stg[1] = make_uint4(codes[4], codes[5], codes[6], codes[7]);
         }
       } else {
+      if (use_res && !mbar_wait(res_full(half), it & 1, abort_flag, status_w, 12)) break;
+      res_seen = it + 1;
 #pragma unroll
       for (int ch = 0; ch < 4; ++ch) {
         uint8_t* slab = smem + L::kStgOff + (half * 2 + (ch >> 1)) * L::kStgSlab + r * 128;
@@ -425,8 +445,18 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
               const float af = magic_ok ? __fsub_rn(__int_as_float(0x4B400000 + a[j]), 12582912.0f) : (float)a[j];
               y[j] = __fmul_rn(__fmul_rn(af, sws[ch * 32 + g * 8 + j]), c);
             }
-            if (residual_p && row_ok && col < n_end) {
-              const uint4 r4 = __ldg(reinterpret_cast<const uint4*>(residual_p + rowoff + col));
+            // where these 8 outputs go in the staging slabs (and where their residual waits)
+            const int chunk = (ch & 1) * 4 + g;          // 16-byte chunk of the slab row; 128-byte swizzle
+            uint4* dst = reinterpret_cast<uint4*>(slab + ((chunk ^ (r & 7)) << 4));
+            bool in_tile = true;
+            if (tn < TN && half == 1 && ch >= 2) {
+              // last slab of a narrower tile: tn - 192 columns, dense rows, no swizzle (its own tensor map)
+              constexpr int tail_bytes = (tn - 192) * 2;
+              in_tile = chunk * 16 < tail_bytes;
+              dst = reinterpret_cast<uint4*>(smem + L::kStgOff + 3 * L::kStgSlab + r * tail_bytes + chunk * 16);
+            }
+            if (use_res && in_tile) {                    // rows and columns outside the matrix arrive as zeros
+              const uint4 r4 = *dst;
               const uint32_t rw[4] = {r4.x, r4.y, r4.z, r4.w};
 #pragma unroll
               for (int j = 0; j < 4; ++j) {
@@ -439,15 +469,7 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             o.y = f32_to_bf16_bits(y[2]) | (f32_to_bf16_bits(y[3]) << 16);
             o.z = f32_to_bf16_bits(y[4]) | (f32_to_bf16_bits(y[5]) << 16);
             o.w = f32_to_bf16_bits(y[6]) | (f32_to_bf16_bits(y[7]) << 16);
-            const int chunk = (ch & 1) * 4 + g;          // 16-byte chunk of the slab row; 128-byte swizzle
-            if (tn < TN && half == 1 && ch >= 2) {
-              // last slab of a narrower tile: tn - 192 columns, dense rows, no swizzle (its own tensor map)
-              constexpr int tail_bytes = (tn - 192) * 2;
-              if (chunk * 16 < tail_bytes)
-                *reinterpret_cast<uint4*>(smem + L::kStgOff + 3 * L::kStgSlab + r * tail_bytes + chunk * 16) = o;
-            } else {
-              *reinterpret_cast<uint4*>(slab + ((chunk ^ (r & 7)) << 4)) = o;
-            }
+            if (in_tile) *dst = o;
           }
         }
       }
@@ -475,6 +497,12 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
       }
     }
     if (issuer) tma_store_wait_read();
+    if (issuer && res_armed > res_seen) {
+      // left the loop on a timeout with a residual load still in flight: bounded wait before the
+      // shared memory it writes to goes away
+      const uint64_t t0 = globaltimer_ns();
+      while (!mbar_try_wait(res_full(half), (uint32_t)(res_armed - 1) & 1u) && globaltimer_ns() - t0 < 2000000ull) {}
+    }
   }
 
   // ------------------------------------------------------------------ teardown
@@ -611,11 +639,17 @@ static int launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, GemmPar
   else tmY = tmA;                                                                  // unused without an output tile
   tmYt = tmY;
   if (kTN < TN && P.Y && !make_out_map(&tmYt, P.Y, P.M, P.N, kTN - 192)) return FPT_ERR_CUDA;
+  CUtensorMap tmR = tmY, tmRt = tmYt;                                              // unused without a residual
+  if (kFuse == 0 && P.Y && P.residual) {
+    if (!make_out_map(&tmR, P.residual, P.M, P.N)) return FPT_ERR_CUDA;
+    tmRt = tmR;
+    if (kTN < TN && !make_out_map(&tmRt, P.residual, P.M, P.N, kTN - 192)) return FPT_ERR_CUDA;
+  }
   P.tiles_m = (P.M + TM - 1) / TM;
   P.num_tiles = P.tiles_m * ((P.N + kTN - 1) / kTN);
   P.kblocks = P.K / BK;
   const int pairs = P.num_tiles < max_pairs ? P.num_tiles : max_pairs;
-  kern<<<2 * pairs, kThreads, L::kAlloc, st>>>(tmA, tmB, tmY, tmYt, P);
+  kern<<<2 * pairs, kThreads, L::kAlloc, st>>>(tmA, tmB, tmY, tmYt, tmR, tmRt, P);
   return cudaGetLastError() == cudaSuccess ? FPT_OK : FPT_ERR_CUDA;
 }
 
