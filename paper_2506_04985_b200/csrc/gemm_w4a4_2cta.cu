@@ -335,6 +335,7 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     const bool magic_ok = kA8 ? P.K < 4096 : P.K <= 32768;   // |acc| < 2^22: int -> float by exponent trick
     const bool issuer = quad == 0 && lane == 0;          // issues the TMA stores (and residual loads) of its half
     const bool use_res = kFuse == 0 && residual_p != nullptr && y_out_p != nullptr;
+    const bool has_z = P.wsum != nullptr;                // asymmetric activation grid: row-sum correction
     int it = 0;
     int res_armed = 0, res_seen = 0;                     // residual loads issued / seen to arrive (tiles, 1-based)
     for (int tile = pair_id; tile < num_tiles; tile += num_pairs, ++it) {
@@ -429,9 +430,21 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
           const int col = nt + half * 128 + ch * 32 + g * 8;
+          // the eight scale factors (and row-sum corrections) of the group as 16-byte shared loads:
+          // every lane reads the same words, one word per load was a wavefront of the contended
+          // shared-memory pipe each
+          const float4 sa = *reinterpret_cast<const float4*>(sws + ch * 32 + g * 8);
+          const float4 sb = *reinterpret_cast<const float4*>(sws + ch * 32 + g * 8 + 4);
+          const float sg[8] = {sa.x, sa.y, sa.z, sa.w, sb.x, sb.y, sb.z, sb.w};
+          int zg[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+          if (has_z) {
+            const int4 za = *reinterpret_cast<const int4*>(zws + ch * 32 + g * 8);
+            const int4 zb = *reinterpret_cast<const int4*>(zws + ch * 32 + g * 8 + 4);
+            zg[0] = za.x; zg[1] = za.y; zg[2] = za.z; zg[3] = za.w; zg[4] = zb.x; zg[5] = zb.y; zg[6] = zb.z; zg[7] = zb.w;
+          }
           int a[8];
 #pragma unroll
-          for (int j = 0; j < 8; ++j) a[j] = (((int)v[ch * 32 + g * 8 + j]) >> kShift) - zws[ch * 32 + g * 8 + j];
+          for (int j = 0; j < 8; ++j) a[j] = (((int)v[ch * 32 + g * 8 + j]) >> kShift) - zg[j];
           if (acc_out_p && row_ok && col < n_end) {
             int4* o = reinterpret_cast<int4*>(acc_out_p + rowoff + col);
             o[0] = make_int4(a[0], a[1], a[2], a[3]);
@@ -443,7 +456,7 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             for (int j = 0; j < 8; ++j) {
               // exact int -> float: 1.5 * 2^23 + a has a in its low mantissa bits
               const float af = magic_ok ? __fsub_rn(__int_as_float(0x4B400000 + a[j]), 12582912.0f) : (float)a[j];
-              y[j] = __fmul_rn(__fmul_rn(af, sws[ch * 32 + g * 8 + j]), c);
+              y[j] = __fmul_rn(__fmul_rn(af, sg[j]), c);
             }
             // where these 8 outputs go in the staging slabs (and where their residual waits)
             const int chunk = (ch & 1) * 4 + g;          // 16-byte chunk of the slab row; 128-byte swizzle
