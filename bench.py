@@ -33,7 +33,7 @@ EPS = 1e-5
 NSETS = 4
 # dram__bytes_read.sum + dram__bytes_write.sum of one fused-QKV matmul launch, from the ncu capture
 # summarised in profiles/gemm_w4a4_pair_2048x6144x4096.md (set to None when the kernel changes)
-GEMM_QKV_DRAM_BYTES = 16.96e6
+GEMM_QKV_DRAM_BYTES = 16.93e6
 METRIC = "W4A4 linear TOPS (prefill, Llama-3-8B-shaped attention projections, 2048 tokens)"
 
 
