@@ -1,8 +1,8 @@
 // Steps (2)+(3) with 8-bit activation codes and 4-bit weights (the W4A8 setting of Sec. 4,
 // Table "4-8-8"): the same exact integer matmul and scale-factor epilogue (App. B, App. J).
 //
-// Large problems use the CTA-pair kernel with the activation tile loaded as int8 (no widening on
-// that side).  Everything else takes a route that needs no kernel of its own: an int8 code is
+// More than 16 tokens and 128 outputs: the CTA-pair kernel with the activation tile loaded as int8 (no
+// widening on that side).  Everything else takes a route that needs no kernel of its own: an int8 code is
 // a = 16 h + l with h = a >> 4 in [-8, 7] and l = a & 15 in [0, 15], so
 //   sum_k a w = 16 sum_k h w + sum_k l w,
 // two 4-bit matmuls (one signed, one unsigned activation operand) through the existing kernels,
@@ -14,7 +14,8 @@ namespace fpt {
 
 static inline size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
 
-static bool a8_uses_pair(int M, int N) { return M > 128 && N > 128; }
+// (below 17 tokens the two register-kernel launches of the split are faster than one pair-kernel launch)
+static bool a8_uses_pair(int M, int N) { return M > 16 && N > 128; }
 
 size_t gemm_a8_scratch_bytes(int M, int N, int K) {
   if (a8_uses_pair(M, N)) return 0;
