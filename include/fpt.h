@@ -211,8 +211,8 @@ int fpt_w4a4_gemm(void* stream, const uint8_t* Xq, const uint8_t* Wq, int M, int
  *   y[t,n]   as in fpt_w4a4_gemm.
  *   Xq8 [M, K] int8;  K % 128 == 0, K <= 16384 (so that (float)acc is exact), N % 8 == 0.
  *   workspace: fpt_workspace_bytes(FPT_OP_GEMM_A8, M, N, K) bytes.
- * More than 16 tokens and 128 outputs: one matmul kernel that loads the activation tile as int8.
- * Smaller problems: the codes are split as a = 16 (a >> 4) + (a & 15) and two 4-bit matmuls are
+ * More than 16 tokens and 128 outputs, or at most 16 tokens: kernels that read the int8 codes as they are.
+ * What is left (more than 16 tokens, at most 128 outputs): the codes are split as a = 16 (a >> 4) + (a & 15) and two 4-bit matmuls are
  * combined exactly in int32 before the scale factors (same result, twice the matmul work).
  */
 int fpt_w4a8_gemm(void* stream, const int8_t* Xq8, const uint8_t* Wq, int M, int N, int K,

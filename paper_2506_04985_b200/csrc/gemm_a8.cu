@@ -2,7 +2,8 @@
 // Table "4-8-8"): the same exact integer matmul and scale-factor epilogue (App. B, App. J).
 //
 // More than 16 tokens and 128 outputs: the CTA-pair kernel with the activation tile loaded as int8 (no
-// widening on that side).  Everything else takes a route that needs no kernel of its own: an int8 code is
+// widening on that side); up to 16 tokens: the register kernel reading int8 codes.  What is left (17 to 128
+// tokens with at most 128 outputs, or more tokens with few outputs) takes a route that needs no kernel of its own: an int8 code is
 // a = 16 h + l with h = a >> 4 in [-8, 7] and l = a & 15 in [0, 15], so
 //   sum_k a w = 16 sum_k h w + sum_k l w,
 // two 4-bit matmuls (one signed, one unsigned activation operand) through the existing kernels,
@@ -14,11 +15,11 @@ namespace fpt {
 
 static inline size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
 
-// (below 17 tokens the two register-kernel launches of the split are faster than one pair-kernel launch)
 static bool a8_uses_pair(int M, int N) { return M > 16 && N > 128; }
+static bool a8_native(int M, int N) { return M <= 16 || a8_uses_pair(M, N); }       // a kernel takes int8 activations as they are
 
 size_t gemm_a8_scratch_bytes(int M, int N, int K) {
-  if (a8_uses_pair(M, N)) return 0;
+  if (a8_native(M, N)) return 0;
   return 2 * up256((size_t)M * K / 2) + 2 * up256((size_t)M * N * 4);
 }
 
@@ -106,11 +107,12 @@ extern "C" int fpt_w4a8_gemm(void* stream, const int8_t* Xq8, const uint8_t* Wq,
   P.sw = sw; P.scale_dtype = scale_dtype;
   P.status = reinterpret_cast<uint32_t*>(workspace);
   P.scratch = ws + kStatusBytes;
-  if (a8_uses_pair(M, N)) {
+  if (a8_native(M, N)) {
     P.a_bits = 8;
     P.act_scale = act_scale; P.post = post;
     P.residual = reinterpret_cast<const __nv_bfloat16*>(residual); P.res_scale = res_scale;
     P.Y = reinterpret_cast<__nv_bfloat16*>(Y); P.acc_out = acc_out;
+    if (M <= 16) return gemm_decode_small_launch(st, reinterpret_cast<const uint8_t*>(Xq8), Wq, P);
     return gemm_pair_launch(st, reinterpret_cast<const uint8_t*>(Xq8), Wq, P);
   }
   // a = 16 h + l through two 4-bit matmuls

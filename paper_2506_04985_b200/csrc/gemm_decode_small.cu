@@ -47,7 +47,19 @@ __device__ __forceinline__ void mma_16x8x32(int (&c)[4], uint32_t a0, uint32_t a
                  : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-template <int NW, int NT, bool kBUnsigned>
+// int8 activation codes (one byte each): 32 codes of a token in the byte order the widening gives the
+// weights (16 even-k codes, then 16 odd-k codes), not multiplied by 16.
+__device__ __forceinline__ void gather_i8(const uint4& lo, const uint4& hi, uint32_t* out) {
+  const uint32_t a[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+#pragma unroll
+  for (int w = 0; w < 4; ++w) {
+    out[w] = __byte_perm(a[2 * w], a[2 * w + 1], 0x6420);
+    out[4 + w] = __byte_perm(a[2 * w], a[2 * w + 1], 0x7531);
+  }
+}
+
+// kA8: Xq holds int8 codes [M, K] instead of packed 4-bit codes [M, K/2] (signed, kBUnsigned = false).
+template <int NW, int NT, bool kBUnsigned, bool kA8 = false>
 __global__ void __launch_bounds__(NW * 32, 768 / (NW * 32)) gemm_w4a4_decode_small_kernel(const uint8_t* __restrict__ Xq,
                                                                           const uint8_t* __restrict__ Wq, const Params D) {
   __shared__ int part[NW][kRows][8 * NT];
@@ -67,7 +79,7 @@ __global__ void __launch_bounds__(NW * 32, 768 / (NW * 32)) gemm_w4a4_decode_sma
   for (int nt = 0; nt < NT; ++nt) {
     const int tok = nt * 8 + g;
     x_ok[nt] = tok < P.M;
-    xr[nt] = Xq + (size_t)(x_ok[nt] ? tok : 0) * row_bytes + 16 * t;
+    xr[nt] = Xq + (size_t)(x_ok[nt] ? tok : 0) * row_bytes * (kA8 ? 2 : 1) + (kA8 ? 32 : 16) * t;
   }
   int acc[NT][4];
 #pragma unroll
@@ -118,9 +130,15 @@ __global__ void __launch_bounds__(NW * 32, 768 / (NW * 32)) gemm_w4a4_decode_sma
         widen(rb_ok ? pb[u] : zero, c);
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
-          const uint4 px = __ldg(reinterpret_cast<const uint4*>(xr[nt] + (size_t)b * 64));
           uint32_t x[8];
-          widen(x_ok[nt] ? px : zero, x);
+          if constexpr (kA8) {
+            const uint4 p0 = __ldg(reinterpret_cast<const uint4*>(xr[nt] + (size_t)b * 128));
+            const uint4 p1 = __ldg(reinterpret_cast<const uint4*>(xr[nt] + (size_t)b * 128 + 16));
+            gather_i8(x_ok[nt] ? p0 : zero, x_ok[nt] ? p1 : zero, x);
+          } else {
+            const uint4 px = __ldg(reinterpret_cast<const uint4*>(xr[nt] + (size_t)b * 64));
+            widen(x_ok[nt] ? px : zero, x);
+          }
 #pragma unroll
           for (int j = 0; j < 4; ++j)
             mma_16x8x32<kBUnsigned>(acc[nt], a[2 * j], c[2 * j], a[2 * j + 1], c[2 * j + 1], x[2 * j], x[2 * j + 1]);
@@ -146,7 +164,7 @@ __global__ void __launch_bounds__(NW * 32, 768 / (NW * 32)) gemm_w4a4_decode_sma
     int s = 0;
 #pragma unroll
     for (int w = 0; w < NW; ++w) s += part[w][o_r][o_tok];
-    const int a = (s >> 8) - o_zw[q];
+    const int a = (s >> (kA8 ? 4 : 8)) - o_zw[q];
     const size_t idx = (size_t)o_tok * P.N + n0 + o_r;
     if (P.acc_out) P.acc_out[idx] = a;
     if (P.Y) {
@@ -160,7 +178,8 @@ __global__ void __launch_bounds__(NW * 32, 768 / (NW * 32)) gemm_w4a4_decode_sma
 template <int NW, int NT>
 static int launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, const Params& D) {
   const int grid = (D.g.N + kRows - 1) / kRows;
-  if (D.g.a_unsigned) gemm_w4a4_decode_small_kernel<NW, NT, true><<<grid, NW * 32, 0, st>>>(Xq, Wq, D);
+  if (D.g.a_bits == 8) gemm_w4a4_decode_small_kernel<NW, NT, false, true><<<grid, NW * 32, 0, st>>>(Xq, Wq, D);
+  else if (D.g.a_unsigned) gemm_w4a4_decode_small_kernel<NW, NT, true><<<grid, NW * 32, 0, st>>>(Xq, Wq, D);
   else gemm_w4a4_decode_small_kernel<NW, NT, false><<<grid, NW * 32, 0, st>>>(Xq, Wq, D);
   return cudaGetLastError() == cudaSuccess ? FPT_OK : FPT_ERR_CUDA;
 }

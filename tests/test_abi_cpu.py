@@ -75,7 +75,7 @@ def test_argument_errors_are_reported_before_any_launch(B):
     assert L.fpt_w4a8_gemm(*a8(4, 64, 128, None, 0)) == B.ERR_WORKSPACE
     assert L.fpt_w4a8_gemm(*a8(4, 64, 128, fake, 16)) == B.ERR_WORKSPACE
     assert L.fpt_workspace_bytes(B.OP_GEMM_A8, 300, 512, 1024) == L.fpt_workspace_bytes(B.OP_GEMM, 300, 512, 1024)
-    assert L.fpt_workspace_bytes(B.OP_GEMM_A8, 16, 512, 1024) > L.fpt_workspace_bytes(B.OP_GEMM, 16, 512, 1024)
+    assert L.fpt_workspace_bytes(B.OP_GEMM_A8, 64, 128, 1024) > L.fpt_workspace_bytes(B.OP_GEMM, 64, 128, 1024)
     qbad = B.QParams(4, False, 0.5, 16)
     r = L.fpt_act_quant(None, fake, 4, 128, 128, ctypes.byref(qbad), B.RMSNORM, 1e-5, None, None, fake, None)
     assert r == B.ERR_BAD_ARG
