@@ -69,3 +69,24 @@ def test_exact_on_small_integers_and_stage_order_is_fixed():
             b[i] = np.float32(a[lo] + a[hi]) if i == lo else np.float32(a[lo] - a[hi])
         a = b
     assert np.array_equal(OH.block_hadamard_f32(x, 8)[0], (a * np.float32(1 / np.sqrt(8.0))).astype(np.float32))
+
+
+def _golden(name):
+    import os
+    path = os.path.join(os.path.dirname(__file__), "golden", name)
+    rows = [ln.split() for ln in open(path) if ln.strip() and not ln.startswith("#")]
+    return np.array(rows, dtype=np.float64)
+
+
+def test_values_the_paper_prints():
+    """tests/golden: the group count and size the paper states for Llama-2 7B's FFN width (App. D), and
+    H_4 written out from the paper's Kronecker definition."""
+    for d, groups, size in _golden("hadamard_groups.txt").astype(np.int64):
+        assert OH.largest_pow2_divisor(int(d)) == size and d // size == groups
+        m = OH.block_hadamard_matrix(int(d))
+        assert m.shape == (d, d)
+        assert np.count_nonzero(m[:size, size:]) == 0 and np.count_nonzero(m[size:2 * size, :size]) == 0   # block diagonal
+    h4 = _golden("hadamard_h4.txt")
+    assert np.array_equal(OH.hadamard_matrix(4) * 2.0, h4)          # the table's factor n^(-1/2) = 1/2 taken out
+    x = np.arange(8, dtype=np.float32).reshape(2, 4)
+    assert np.array_equal(OH.block_hadamard_f32(x), (x.astype(np.float64) @ h4.T * 0.5).astype(np.float32))
