@@ -16,11 +16,15 @@
 // Roles per CTA (20 warps):
 //   warp 0        TMA producer: packed tiles (128 rows x 64 bytes of each operand per k-block)
 //   warp 1        tensor-memory owner; in the leader CTA (rank 0) also the MMA issuer
-//   warps 4..7    activation converters: shared -> registers -> widen -> tcgen05.st (one row per thread)
-//   warps 8..11   weight converters: shared -> widen -> 128-byte-swizzled K-major int8 tile
+//   warps 4..7    activation converters: shared -> registers -> widen -> tcgen05.st (one row per thread);
+//                 while that store completes they also widen the last quarter of the weight tile
+//   warps 8..11   weight converters: shared -> widen -> 128-byte-swizzled K-major int8 tile (three quarters)
 //   warps 12..19  epilogue: tcgen05.ld, >> 8, scales, bf16 into a swizzled shared-memory tile; the
-//                 accumulator is released as soon as it has been read, the tile leaves by TMA store
+//                 accumulator is released as soon as it has been read, the tile leaves by TMA store;
+//                 a residual tile is fetched by TMA into the same slabs while the tile's matmul runs
 // Both operands are widened as code*16 (see gemm_w4a4.cu), so the accumulator holds 256 * sum.
+// Variants (template parameters): the two fused SwiGLU epilogues, int8 activation codes (the
+// activation tile then needs no widening and the shift is 4), output tiles of 208..256 columns.
 #include <cuda.h>
 
 #include "fpt_internal.cuh"
