@@ -26,7 +26,7 @@ struct ActQuantParams {
 
 // T threads per token, up to V 16-byte chunks (8 elements) per thread held in registers.
 template <int T, int V>
-__global__ void __launch_bounds__(T, 2048 / T) act_quant_kernel(const ActQuantParams P) {
+__global__ void __launch_bounds__(T, V <= 4 ? 2048 / T : 1) act_quant_kernel(const ActQuantParams P) {
   __shared__ double warp_part[T / 32];
   __shared__ float  bcast;
   const int t = blockIdx.x;

@@ -54,7 +54,7 @@ __device__ __forceinline__ uint2 quant8_chunk(const uint4& v, float p, float inv
 }
 
 template <int T, int V, int BITS>
-__global__ void __launch_bounds__(T, 2048 / T) act_quant_dyn_kernel(const DynQuantParams P) {
+__global__ void __launch_bounds__(T, V <= 4 ? 2048 / T : 1) act_quant_dyn_kernel(const DynQuantParams P) {
   __shared__ double warp_part[T / 32];
   __shared__ uint32_t warp_max[T / 32];
   __shared__ float bcast;
