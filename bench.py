@@ -422,6 +422,13 @@ def run_gpu(args):
             torch.cuda.empty_cache()
             var[name] = {"us": us, "TOP/s": ops / us / 1e6}
         other["variants on 2048x6144x4096 (quantise + matmul)"] = var
+        # the attention block's two halves around the caller's attention (scaler at the attention output,
+        # normalised residual added in the output projection's epilogue)
+        runs, ops, _ = MB.make_case("attn_proj", M_TOK, N_QKV, HID, 4, dev)
+        us = MB.time_case_graph(runs, 20)
+        del runs
+        torch.cuda.empty_cache()
+        other["attention block projections with residual, 2048 tokens (4 kernels)"] = {"us": us, "TOP/s": ops / us / 1e6}
 
     if rank == 0:
         rows = M_TOK

@@ -6,6 +6,7 @@
     python -m paper_2506_04985_b200.microbench linear    --M 64 --N 14336 --K 4096
     python -m paper_2506_04985_b200.microbench hadamard_quant --M 4096 --K 14336
     python -m paper_2506_04985_b200.microbench mlp       --M 4096 --K 4096 --N 14336      (mlp_hadamard: with the online transform)
+    python -m paper_2506_04985_b200.microbench attn_proj --M 2048 --N 6144 --K 4096       (QKV and output projections with the residual)
     python -m paper_2506_04985_b200.microbench gemm_a8   --M 2048 --N 6144 --K 4096       (int8 activation codes)
     python -m paper_2506_04985_b200.microbench linear_dynamic --M 2048 --N 6144 --K 4096 --bits 4
     python -m paper_2506_04985_b200.microbench act_quant_dynamic --M 2048 --K 4096 --bits 4
@@ -103,6 +104,22 @@ def make_case(kind, M, N, K, sets, dev, f16_scales=False, bits=4):
             runs.append(lambda x=x, wq=wq, sw=sw, y=y, ws=ws: B.fpt_w4a4_linear(
                 x, wq, sw, qp, B.RMSNORM, 1e-5, want_s_out=False, ws=ws, Y=y))
         return runs, 2.0 * M * N * K, 2.0 * M * K + N * K / 2 + N * ssz + 2.0 * M * N
+    if kind == "attn_proj":                 # K = d (= query width), N = fused QKV width; both halves of the attention block
+        d, nqkv = K, N
+        for _ in range(sets):
+            x, a = _bf16(M, d, dev), _bf16(M, d, dev)          # a stands for the caller's attention output
+            wqkv, wo = _codes(nqkv, d // 2, dev), _codes(d, d // 2, dev)
+            sqkv = torch.rand((nqkv,), device=dev).to(sdt) * 0.01 + 0.001
+            so = torch.rand((d,), device=dev).to(sdt) * 0.01 + 0.001
+            qkv = torch.empty((M, nqkv), dtype=torch.bfloat16, device=dev)
+            y = torch.empty((M, d), dtype=torch.bfloat16, device=dev)
+            ws = B.new_workspace(B.OP_LINEAR, M, max(nqkv, d), d, dev)
+
+            def run(x=x, a=a, wqkv=wqkv, wo=wo, sqkv=sqkv, so=so, qkv=qkv, y=y, ws=ws):
+                _, s_n, r = B.fpt_decoder_attn_qkv(x, wqkv, sqkv, qp, 1e-5, ws=ws, QKV=qkv)
+                B.fpt_decoder_attn_out(a, wo, so, qp, s_n, X=x, r=r, ws=ws, Y=y)
+            runs.append(run)
+        return runs, 2.0 * M * d * (nqkv + d), 6.0 * M * d + (nqkv + d) * d / 2 + 2.0 * M * nqkv + 2.0 * M * d
     if kind in ("mlp", "mlp_hadamard"):    # K = d, N = d_ff
         d, dff = K, N
         for _ in range(sets):
@@ -155,7 +172,7 @@ def time_case_graph(runs, reps, warmup=3, replays=5):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("kind", choices=["gemm", "act_quant", "silu_quant", "hadamard_quant", "linear", "mlp", "mlp_hadamard",
-                                     "gemm_a8", "act_quant_dynamic", "linear_dynamic"])
+                                     "gemm_a8", "act_quant_dynamic", "linear_dynamic", "attn_proj"])
     ap.add_argument("--M", type=int, default=2048)
     ap.add_argument("--N", type=int, default=4096)
     ap.add_argument("--K", type=int, default=4096)
