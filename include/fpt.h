@@ -78,6 +78,7 @@ extern "C" {
 #define FPT_OP_GEMM   2
 #define FPT_OP_GEMM_A8   3     /* fpt_w4a8_gemm                                   */
 #define FPT_OP_LINEAR_A8 4     /* fpt_w4a4_linear / _dynamic with 8-bit activations */
+#define FPT_OP_MLP_HADAMARD 5  /* fpt_decoder_mlp with mid_hadamard = 1              */
 
 /* One quantiser, as the paper parametrises it: bit-width, grid kind, static scale and
  * offset (App. D "General set-up"). HOST struct. */
@@ -91,6 +92,16 @@ typedef struct fpt_qparams {
 
 int         fpt_version(void);
 const char* fpt_strerror(int code);
+
+/*
+ * Kernels of steps (1)-(3) are launched so that each may start (set up its barriers and tensor
+ * memory, and wait) while the kernel before it in the stream is still draining; each orders itself
+ * behind that kernel before it touches any operand, so results and stream semantics are unchanged
+ * (no counterpart in the paper: a launch mode).  enabled = 0 switches back to plain launches for
+ * every later call of the process, e.g. under a tool that does not follow such launches.
+ * Returns the previous setting.  Not synchronised with concurrent calls of the other entry points.
+ */
+int fpt_set_programmatic_launch(int enabled);
 
 /*
  * Offline weight quantiser (uniform grid, round-to-nearest, per-output-channel scale;
@@ -293,7 +304,10 @@ int fpt_w4a4_linear_static(void* stream, const void* X, int M, int K,
  *   Wgu_q [2 d_ff, d/2] and sw_gu [2 d_ff] in the layout of fpt_interleave_gate_up;
  *   Wd_q [d, d_ff/2], sw_d [d]; s_prev [M] or NULL (= 1); s_out [M] or NULL.
  *   d % 128 == 0, d_ff % 128 == 0.  Both grids symmetric in this version.
- *   workspace: fpt_workspace_bytes(FPT_OP_MLP, M, d_ff, d) bytes.
+ *   workspace: fpt_workspace_bytes(FPT_OP_MLP, M, d_ff, d) bytes, or (FPT_OP_MLP_HADAMARD, M, d_ff, d)
+ *   with mid_hadamard = 1.  A 16-bit buffer between the two matmuls is part of it only where a route
+ *   uses one: none with more than 128 tokens and no transform (the gate||up matmul quantises the
+ *   products itself), the products [M, d_ff] with the transform, gate||up [M, 2 d_ff] up to 128 tokens.
  */
 int fpt_decoder_mlp(void* stream, const void* X, int M, int d, int d_ff,
                     const uint8_t* Wgu_q, const void* sw_gu, const uint8_t* Wd_q, const void* sw_d,
@@ -332,6 +346,22 @@ int fpt_decoder_attn_out(void* stream, const void* A, int M, int k_o,
                          const uint8_t* Wo_q, const void* sw_o, int scale_dtype, const int32_t* wsum_o, int d,
                          const fpt_qparams* qp_ap, const float* s_n, const void* X, const float* r,
                          void* Y, void* workspace, size_t workspace_bytes);
+
+/*
+ * Measurement aid; the paper has no counterpart.  Runs nothing of the path: one thread per CTA
+ * (pair = 0) or per pair of CTAs (pair = 1, `ctas` even) issues 4 * iters 8-bit integer
+ * tensor-core instructions of 128 (pair: 256) rows x n columns x 32 codes on operand tiles that
+ * never move, rotating over n_acc accumulators (n_acc * n <= 480), with the row operand read
+ * from tensor memory (a_in_tmem = 1) or from shared memory.  2 * rows * n * 32 * 4 * iters * CTAs
+ * (pairs) integer operations per launch; the rate it reaches is the ceiling the matmul kernels
+ * are compared with.
+ *   n       multiple of 16 in [16, 256]
+ *   cycles  device [ctas] (pair: [ctas / 2]) out, may be NULL: SM clock ticks from the first issue
+ *           to the completion of the last instruction
+ *   workspace  device, 16-byte aligned, at least 8192 bytes: status block (fpt_check_status)
+ */
+int fpt_probe_mma(void* stream, int pair, int n, int n_acc, int a_in_tmem, int iters, int ctas,
+                  unsigned long long* cycles, void* workspace);
 
 /* Bytes of caller-provided scratch an entry point needs (op = FPT_OP_*).
  * FPT_OP_LINEAR / FPT_OP_GEMM / FPT_OP_GEMM_A8 / FPT_OP_LINEAR_A8: (M, N, K); FPT_OP_MLP: (M, d_ff, d). */

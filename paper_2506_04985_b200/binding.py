@@ -19,13 +19,13 @@ DTYPE_BF16, DTYPE_F32, DTYPE_F16 = 0, 1, 2
 RANGE_MINMAX, RANGE_LP = 0, 1
 RMSNORM, SCALE_INPUT, SILU_MUL, GU_INTERLEAVED = 1, 2, 4, 8
 POST_NONE, POST_INVERSE_OF_PRE, POST_VECTOR = 0, 1, 2
-OP_LINEAR, OP_MLP, OP_GEMM, OP_GEMM_A8, OP_LINEAR_A8 = 0, 1, 2, 3, 4
+OP_LINEAR, OP_MLP, OP_GEMM, OP_GEMM_A8, OP_LINEAR_A8, OP_MLP_HADAMARD = 0, 1, 2, 3, 4, 5
 
 EXPORTS = ["fpt_version", "fpt_strerror", "fpt_quantize_weights", "fpt_interleave_gate_up", "fpt_act_quant", "fpt_hadamard_quant",
            "fpt_w4a4_gemm", "fpt_w4a4_linear", "fpt_w4a4_linear_static", "fpt_decoder_mlp", "fpt_decoder_attn_qkv",
            "fpt_decoder_attn_out", "fpt_act_quant_dynamic", "fpt_w4a4_linear_dynamic", "fpt_w4a8_gemm", "fpt_workspace_bytes",
            "fpt_reset_status",
-           "fpt_check_status"]
+           "fpt_check_status", "fpt_probe_mma", "fpt_set_programmatic_launch"]
 
 
 class QParams(ctypes.Structure):
@@ -44,6 +44,20 @@ class FptError(RuntimeError):
 
 
 _lib = None
+_allocator = None
+
+
+def set_allocator(fn):
+    """Routes every device allocation of this module through `fn(shape, dtype, device) -> tensor`
+    (None: plain torch.empty).  The GPU tests install one that surrounds each buffer with guard bands."""
+    global _allocator
+    _allocator = fn
+
+
+def _empty(shape, dtype, device):
+    if _allocator is not None:
+        return _allocator(shape, dtype, device)
+    return torch.empty(shape, dtype=dtype, device=device)
 
 
 def lib():
@@ -75,6 +89,8 @@ def lib():
         L.fpt_workspace_bytes.argtypes = [ci, ci, ci, ci]
         L.fpt_reset_status.argtypes = [vp, vp]
         L.fpt_check_status.argtypes = [vp, vp]
+        L.fpt_set_programmatic_launch.argtypes = [ci]
+        L.fpt_probe_mma.argtypes = [vp, ci, ci, ci, ci, ci, ci, vp, vp]
         for name in EXPORTS:
             if name not in ("fpt_strerror", "fpt_workspace_bytes", "fpt_version"):
                 getattr(L, name).restype = ci
@@ -113,7 +129,7 @@ def fpt_workspace_bytes(op, M, N, K):
 
 def new_workspace(op, M, N, K, device="cuda"):
     """Allocates a workspace of the required size and clears its status word."""
-    ws = torch.empty(max(fpt_workspace_bytes(op, M, N, K), 256), dtype=torch.uint8, device=device)
+    ws = _empty(max(fpt_workspace_bytes(op, M, N, K), 256), dtype=torch.uint8, device=device)
     _check(lib().fpt_reset_status(_stream(), _ptr(ws)), "fpt_reset_status")
     return ws
 
@@ -126,9 +142,9 @@ def fpt_quantize_weights(W, qp=None, range_mode=RANGE_MINMAX, p=3.0, scale_dtype
     """W [N, K] bf16/f32 -> (Wq uint8 [N, K/2], sw [N], wsum int32 [N] or None)."""
     qp = qp or QParams()
     N, K = W.shape
-    Wq = torch.empty((N, K // 2), dtype=torch.uint8, device=W.device)
-    sw = torch.empty((N,), dtype=scale_dtype, device=W.device)
-    wsum = torch.empty((N,), dtype=torch.int32, device=W.device) if want_wsum else None
+    Wq = _empty((N, K // 2), dtype=torch.uint8, device=W.device)
+    sw = _empty((N,), dtype=scale_dtype, device=W.device)
+    wsum = _empty((N,), dtype=torch.int32, device=W.device) if want_wsum else None
     wd = {torch.bfloat16: DTYPE_BF16, torch.float32: DTYPE_F32}[W.dtype]
     _check(lib().fpt_quantize_weights(_stream(), _ptr(W), wd, N, K, ctypes.byref(qp), range_mode, p,
                                       _scale_dtype(sw), _ptr(Wq), _ptr(sw), _ptr(wsum)), "fpt_quantize_weights")
@@ -137,8 +153,8 @@ def fpt_quantize_weights(W, qp=None, range_mode=RANGE_MINMAX, p=3.0, scale_dtype
 
 def fpt_interleave_gate_up(Wg_q, Wu_q, sw_g, sw_u):
     d_ff, kb = Wg_q.shape
-    Wgu = torch.empty((2 * d_ff, kb), dtype=torch.uint8, device=Wg_q.device)
-    sw = torch.empty((2 * d_ff,), dtype=sw_g.dtype, device=Wg_q.device)
+    Wgu = _empty((2 * d_ff, kb), dtype=torch.uint8, device=Wg_q.device)
+    sw = _empty((2 * d_ff,), dtype=sw_g.dtype, device=Wg_q.device)
     _check(lib().fpt_interleave_gate_up(_stream(), _ptr(Wg_q), _ptr(Wu_q), _ptr(sw_g), _ptr(sw_u),
                                         _scale_dtype(sw_g), d_ff, kb * 2, _ptr(Wgu), _ptr(sw)),
            "fpt_interleave_gate_up")
@@ -153,10 +169,10 @@ def fpt_act_quant(X, qp, flags=RMSNORM, eps=1e-5, X2=None, s_in=None, K=None, wa
     if out is not None:
         Xq = out
     elif qp.bits == 8:
-        Xq = torch.empty((M, K), dtype=torch.int8, device=X.device)
+        Xq = _empty((M, K), dtype=torch.int8, device=X.device)
     else:
-        Xq = torch.empty((M, K // 2), dtype=torch.uint8, device=X.device)
-    s_out = torch.empty((M,), dtype=torch.float32, device=X.device) if want_s_out else None
+        Xq = _empty((M, K // 2), dtype=torch.uint8, device=X.device)
+    s_out = _empty((M,), dtype=torch.float32, device=X.device) if want_s_out else None
     _check(lib().fpt_act_quant(_stream(), _ptr(X), M, K, ldx, ctypes.byref(qp), flags, eps, _ptr(X2), _ptr(s_in),
                                _ptr(Xq), _ptr(s_out)), "fpt_act_quant")
     return Xq, s_out
@@ -171,8 +187,8 @@ def fpt_w4a4_gemm(Xq, Wq, sw, act_scale, wsum=None, act_symmetric=True, act_zero
     if ws is None:
         ws = new_workspace(OP_GEMM, M, N, K, Xq.device)
     if Y is None and want_y:
-        Y = torch.empty((M, N), dtype=torch.bfloat16, device=Xq.device)
-    acc = torch.empty((M, N), dtype=torch.int32, device=Xq.device) if want_acc else None
+        Y = _empty((M, N), dtype=torch.bfloat16, device=Xq.device)
+    acc = _empty((M, N), dtype=torch.int32, device=Xq.device) if want_acc else None
     _check(lib().fpt_w4a4_gemm(_stream(), _ptr(Xq), _ptr(Wq), M, N, K, _ptr(sw), _scale_dtype(sw), _ptr(wsum),
                                float(act_scale), int(bool(act_symmetric)), int(act_zero_point), _ptr(post),
                                _ptr(residual), _ptr(res_scale), _ptr(Y), _ptr(acc), _ptr(ws), ws.numel()),
@@ -188,8 +204,8 @@ def fpt_w4a4_linear(X, Wq, sw, qp, flags=RMSNORM, eps=1e-5, s_in=None, post_mode
     if ws is None:
         ws = new_workspace(OP_LINEAR_A8 if qp.bits == 8 else OP_LINEAR, M, N, K, X.device)
     if Y is None:
-        Y = torch.empty((M, N), dtype=torch.bfloat16, device=X.device)
-    s_out = torch.empty((M,), dtype=torch.float32, device=X.device) if want_s_out else None
+        Y = _empty((M, N), dtype=torch.bfloat16, device=X.device)
+    s_out = _empty((M,), dtype=torch.float32, device=X.device) if want_s_out else None
     _check(lib().fpt_w4a4_linear(_stream(), _ptr(X), M, K, _ptr(Wq), _ptr(sw), _scale_dtype(sw), _ptr(wsum), N,
                                  ctypes.byref(qp), flags, eps, _ptr(s_in), post_mode, _ptr(post), _ptr(Y),
                                  _ptr(s_out), _ptr(ws), ws.numel()), "fpt_w4a4_linear")
@@ -218,7 +234,7 @@ def fpt_hadamard_quant(X, qp, flags=SCALE_INPUT, s_in=None, K=None, out=None):
     M, ldx = X.shape
     if K is None:
         K = ldx // 2 if (flags & GU_INTERLEAVED) else ldx
-    Xq = out if out is not None else torch.empty((M, K // 2), dtype=torch.uint8, device=X.device)
+    Xq = out if out is not None else _empty((M, K // 2), dtype=torch.uint8, device=X.device)
     _check(lib().fpt_hadamard_quant(_stream(), _ptr(X), M, K, ldx, ctypes.byref(qp), flags, _ptr(s_in), _ptr(Xq)),
            "fpt_hadamard_quant")
     return Xq
@@ -230,10 +246,10 @@ def fpt_decoder_mlp(X, Wgu_q, sw_gu, Wd_q, sw_d, qp_in, qp_mid, eps=1e-5, s_prev
     M, d = X.shape
     d_ff = Wgu_q.shape[0] // 2
     if ws is None:
-        ws = new_workspace(OP_MLP, M, d_ff, d, X.device)
+        ws = new_workspace(OP_MLP_HADAMARD if mid_hadamard else OP_MLP, M, d_ff, d, X.device)
     if Y is None:
-        Y = torch.empty((M, d), dtype=torch.bfloat16, device=X.device)
-    s_out = torch.empty((M,), dtype=torch.float32, device=X.device) if want_s_out else None
+        Y = _empty((M, d), dtype=torch.bfloat16, device=X.device)
+    s_out = _empty((M,), dtype=torch.float32, device=X.device) if want_s_out else None
     _check(lib().fpt_decoder_mlp(_stream(), _ptr(X), M, d, d_ff, _ptr(Wgu_q), _ptr(sw_gu), _ptr(Wd_q), _ptr(sw_d),
                                  _scale_dtype(sw_gu), ctypes.byref(qp_in), ctypes.byref(qp_mid), eps, _ptr(s_prev),
                                  _ptr(s_out), int(bool(add_residual)), int(bool(mid_hadamard)), _ptr(Y), _ptr(ws),
@@ -249,9 +265,9 @@ def fpt_decoder_attn_qkv(X, Wqkv_q, sw_qkv, qp_in, eps=1e-5, s_prev=None, wsum=N
     if ws is None:
         ws = new_workspace(OP_LINEAR, M, n_qkv, d, X.device)
     if QKV is None:
-        QKV = torch.empty((M, n_qkv), dtype=torch.bfloat16, device=X.device)
-    s_out = torch.empty((M,), dtype=torch.float32, device=X.device)
-    r_out = torch.empty((M,), dtype=torch.float32, device=X.device)
+        QKV = _empty((M, n_qkv), dtype=torch.bfloat16, device=X.device)
+    s_out = _empty((M,), dtype=torch.float32, device=X.device)
+    r_out = _empty((M,), dtype=torch.float32, device=X.device)
     _check(lib().fpt_decoder_attn_qkv(_stream(), _ptr(X), M, d, _ptr(Wqkv_q), _ptr(sw_qkv), _scale_dtype(sw_qkv),
                                       _ptr(wsum), n_qkv, ctypes.byref(qp_in), eps, _ptr(s_prev), _ptr(s_out),
                                       _ptr(r_out), _ptr(QKV), _ptr(ws), ws.numel()), "fpt_decoder_attn_qkv")
@@ -266,7 +282,7 @@ def fpt_decoder_attn_out(A, Wo_q, sw_o, qp_ap, s_n, X=None, r=None, wsum=None, w
     if ws is None:
         ws = new_workspace(OP_LINEAR, M, d, k_o, A.device)
     if Y is None:
-        Y = torch.empty((M, d), dtype=torch.bfloat16, device=A.device)
+        Y = _empty((M, d), dtype=torch.bfloat16, device=A.device)
     _check(lib().fpt_decoder_attn_out(_stream(), _ptr(A), M, k_o, _ptr(Wo_q), _ptr(sw_o), _scale_dtype(sw_o), _ptr(wsum),
                                       d, ctypes.byref(qp_ap), _ptr(s_n), _ptr(X), _ptr(r), _ptr(Y), _ptr(ws),
                                       ws.numel()), "fpt_decoder_attn_out")
@@ -277,10 +293,10 @@ def fpt_act_quant_dynamic(X, bits=4, flags=RMSNORM, eps=1e-5, s_in=None, want_s_
     """Dynamic per-token grid -> (codes uint8 [M, K/2] or int8 [M, K], s_out f32 [M] or None, delta f32 [M])."""
     M, K = X.shape
     if out is None:
-        out = (torch.empty((M, K // 2), dtype=torch.uint8, device=X.device) if bits == 4
-               else torch.empty((M, K), dtype=torch.int8, device=X.device))
-    s_out = torch.empty((M,), dtype=torch.float32, device=X.device) if want_s_out else None
-    delta = torch.empty((M,), dtype=torch.float32, device=X.device)
+        out = (_empty((M, K // 2), dtype=torch.uint8, device=X.device) if bits == 4
+               else _empty((M, K), dtype=torch.int8, device=X.device))
+    s_out = _empty((M,), dtype=torch.float32, device=X.device) if want_s_out else None
+    delta = _empty((M,), dtype=torch.float32, device=X.device)
     _check(lib().fpt_act_quant_dynamic(_stream(), _ptr(X), M, K, X.stride(0), bits, flags, eps, _ptr(s_in), _ptr(out),
                                        _ptr(s_out), _ptr(delta)), "fpt_act_quant_dynamic")
     return out, s_out, delta
@@ -294,8 +310,8 @@ def fpt_w4a4_linear_dynamic(X, Wq, sw, bits=4, flags=RMSNORM, eps=1e-5, s_in=Non
     if ws is None:
         ws = new_workspace(OP_LINEAR_A8 if bits == 8 else OP_LINEAR, M, N, K, X.device)
     if Y is None:
-        Y = torch.empty((M, N), dtype=torch.bfloat16, device=X.device)
-    s_out = torch.empty((M,), dtype=torch.float32, device=X.device) if want_s_out else None
+        Y = _empty((M, N), dtype=torch.bfloat16, device=X.device)
+    s_out = _empty((M,), dtype=torch.float32, device=X.device) if want_s_out else None
     _check(lib().fpt_w4a4_linear_dynamic(_stream(), _ptr(X), M, K, _ptr(Wq), _ptr(sw), _scale_dtype(sw), N, bits, flags,
                                          eps, _ptr(s_in), post_mode, _ptr(post), _ptr(Y), _ptr(s_out), _ptr(ws),
                                          ws.numel()), "fpt_w4a4_linear_dynamic")
@@ -310,9 +326,25 @@ def fpt_w4a8_gemm(Xq8, Wq, sw, act_scale, post=None, residual=None, res_scale=No
     if ws is None:
         ws = new_workspace(OP_GEMM_A8, M, N, K, Xq8.device)
     if Y is None and want_y:
-        Y = torch.empty((M, N), dtype=torch.bfloat16, device=Xq8.device)
-    acc = torch.empty((M, N), dtype=torch.int32, device=Xq8.device) if want_acc else None
+        Y = _empty((M, N), dtype=torch.bfloat16, device=Xq8.device)
+    acc = _empty((M, N), dtype=torch.int32, device=Xq8.device) if want_acc else None
     _check(lib().fpt_w4a8_gemm(_stream(), _ptr(Xq8), _ptr(Wq), M, N, K, _ptr(sw), _scale_dtype(sw), float(act_scale),
                                _ptr(post), _ptr(residual), _ptr(res_scale), _ptr(Y), _ptr(acc), _ptr(ws), ws.numel()),
            "fpt_w4a8_gemm")
     return Y, acc
+
+
+def fpt_probe_mma(pair, n, n_acc, a_in_tmem, iters, ctas, ws=None, want_cycles=True):
+    """Measurement aid: bare 8-bit integer tensor-core instructions (see fpt.h) -> cycles uint64 per CTA (pair) or None."""
+    dev = torch.device("cuda", torch.cuda.current_device())
+    if ws is None:
+        ws = torch.zeros((8192,), dtype=torch.uint8, device=dev)
+    cyc = torch.zeros((ctas // 2 if pair else ctas,), dtype=torch.int64, device=dev) if want_cycles else None
+    _check(lib().fpt_probe_mma(_stream(), int(pair), n, n_acc, int(a_in_tmem), iters, ctas, _ptr(cyc), _ptr(ws)),
+           "fpt_probe_mma")
+    return cyc
+
+
+def fpt_set_programmatic_launch(enabled):
+    """Switches programmatic dependent launch of the library's kernels on or off; returns the previous setting."""
+    return lib().fpt_set_programmatic_launch(int(bool(enabled)))

@@ -29,6 +29,8 @@ template <int T, int V>
 __global__ void __launch_bounds__(T, V <= 4 ? 2048 / T : 1) act_quant_kernel(const ActQuantParams P) {
   __shared__ double warp_part[T / 32];
   __shared__ float  bcast;
+  pdl_wait();                                    // X may come from the kernel before this one
+  pdl_launch_dependents();
   const int t = blockIdx.x;
   const int tid = threadIdx.x;
   const int chunks = P.K >> 3;                   // 16-byte chunks per row
@@ -117,6 +119,8 @@ __global__ void __launch_bounds__(T, V <= 4 ? 2048 / T : 1) act_quant_kernel(con
 // reduction is a warp shuffle, no shared memory and no block-wide barrier.  W warps per CTA.
 template <int V, int W>
 __global__ void __launch_bounds__(W * 32) act_quant_warp_kernel(const ActQuantParams P) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int lane = threadIdx.x & 31;
   const int t = blockIdx.x * W + (threadIdx.x >> 5);
   if (t >= P.M) return;
@@ -183,6 +187,8 @@ __global__ void __launch_bounds__(1024) act_quant_stream_kernel(const ActQuantPa
   if (lane == 0) { mbar_init(bars, 1); mbar_init(bars + 8, 1); }
   fence_mbar_init();
   __syncthreads();
+  pdl_wait();
+  pdl_launch_dependents();
   const int chunks = P.K >> 3;
   const long long stride = (long long)gridDim.x * W;
   const long long first = (long long)warp * gridDim.x + blockIdx.x;
@@ -252,15 +258,9 @@ __global__ void __launch_bounds__(1024) act_quant_stream_kernel(const ActQuantPa
 }
 
 static cudaError_t launch_stream(const ActQuantParams& P, cudaStream_t st) {
-  static int sms = 0;
-  if (!sms) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (sms <= 0) sms = 1;
-    cudaError_t e = cudaFuncSetAttribute(act_quant_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
-    if (e != cudaSuccess) { sms = 0; return e; }
-  }
+  static PerDeviceInt attr_set;
+  if (!ensure_smem_attr(attr_set, act_quant_stream_kernel, 220 * 1024)) return cudaErrorInvalidValue;
+  const int sms = device_sm_count();
   // as many warps as row buffers fit (each warp needs at least one); two buffers per warp when
   // 32 warps leave room for them
   const uint32_t row_bytes = (uint32_t)P.K * 2;
@@ -279,20 +279,17 @@ static cudaError_t launch_stream(const ActQuantParams& P, cudaStream_t st) {
     if (eff > best + 0.1) { best = eff; W = w; }
   }
   const size_t smem = (size_t)W * NB * row_bytes + (size_t)W * 16;
-  act_quant_stream_kernel<<<grid, W * 32, smem, st>>>(P, W, NB, row_bytes);
-  return cudaGetLastError();
+  return launch_kernel(act_quant_stream_kernel, dim3(grid), dim3(W * 32), smem, st, true, P, W, NB, row_bytes);
 }
 
 template <int V, int W>
 static cudaError_t launch_warp(const ActQuantParams& P, cudaStream_t st) {
-  act_quant_warp_kernel<V, W><<<(P.M + W - 1) / W, W * 32, 0, st>>>(P);
-  return cudaGetLastError();
+  return launch_kernel(act_quant_warp_kernel<V, W>, dim3((P.M + W - 1) / W), dim3(W * 32), 0, st, true, P);
 }
 
 template <int T, int V>
 static cudaError_t launch(const ActQuantParams& P, cudaStream_t st) {
-  act_quant_kernel<T, V><<<P.M, T, 0, st>>>(P);
-  return cudaGetLastError();
+  return launch_kernel(act_quant_kernel<T, V>, dim3(P.M), dim3(T), 0, st, true, P);
 }
 
 // Internal entry shared by the public functions (also fills post_inv / r_out for the

@@ -59,6 +59,8 @@ __global__ void __launch_bounds__(T, V <= 4 ? 2048 / T : 1) act_quant_dyn_kernel
   __shared__ uint32_t warp_max[T / 32];
   __shared__ float bcast;
   __shared__ uint32_t bmax;
+  pdl_wait();                                    // X may come from the kernel before this one
+  pdl_launch_dependents();
   const int t = blockIdx.x, tid = threadIdx.x;
   const int chunks = P.K >> 3;
   const size_t row = (size_t)t * (size_t)(P.ldx >> 3);
@@ -158,9 +160,8 @@ __global__ void __launch_bounds__(T, V <= 4 ? 2048 / T : 1) act_quant_dyn_kernel
 
 template <int T, int V>
 static cudaError_t launch(const DynQuantParams& P, int bits, cudaStream_t st) {
-  if (bits == 8) act_quant_dyn_kernel<T, V, 8><<<P.M, T, 0, st>>>(P);
-  else act_quant_dyn_kernel<T, V, 4><<<P.M, T, 0, st>>>(P);
-  return cudaGetLastError();
+  if (bits == 8) return launch_kernel(act_quant_dyn_kernel<T, V, 8>, dim3(P.M), dim3(T), 0, st, true, P);
+  return launch_kernel(act_quant_dyn_kernel<T, V, 4>, dim3(P.M), dim3(T), 0, st, true, P);
 }
 
 // bits 4: dynamic only (the static 4-bit grid has its own kernels); bits 8: static (dynamic = 0,

@@ -14,17 +14,77 @@ static int check_qp(const fpt_qparams* qp) {
   return FPT_OK;
 }
 
+// bf16 buffer between the two matmuls of the MLP block: nothing when the gate||up matmul's epilogue
+// quantises the products itself (more than 128 tokens, no online transform), the products [M, d_ff]
+// when the transform needs whole rows of them, gate||up [M, 2 d_ff] on the unfused route.
+static size_t mlp_gu_bytes(int M, int d_ff, bool hadamard) {
+  if (M > 128) return hadamard ? (size_t)M * (size_t)d_ff * 2 : 0;
+  return (size_t)M * 2 * (size_t)d_ff * 2;
+}
+
 static int check_gemm_shape(int M, int N, int K) {
   if (M <= 0 || N <= 0 || K <= 0) return FPT_ERR_BAD_ARG;
   if (K % 128 != 0 || K > 65535 || N % 8 != 0) return FPT_ERR_UNSUPPORTED;
   return FPT_OK;
 }
 
+static int g_programmatic_launch = 1;
+int programmatic_launch_enabled() { return g_programmatic_launch; }
+
+// The 4-bit static linear behind fpt_w4a4_linear and fpt_w4a4_linear_static: one set of argument
+// checks and one carving of the workspace (control block | matmul scratch | codes | one float per token).
+int linear4_check(const void* X, const uint8_t* Wq, const void* sw, int scale_dtype, const int32_t* wsum, const void* Y,
+                  const fpt_qparams* act_qp, int M, int N, int K, int flags, const float* s_in, int post_mode,
+                  const float* post) {
+  if (!X || !Wq || !sw || !Y) return FPT_ERR_BAD_ARG;
+  int rc = check_qp(act_qp);
+  if (rc) return rc;
+  rc = check_gemm_shape(M, N, K);
+  if (rc) return rc;
+  if (scale_dtype != FPT_DTYPE_F32 && scale_dtype != FPT_DTYPE_F16) return FPT_ERR_BAD_ARG;
+  if (flags & ~(FPT_RMSNORM | FPT_SCALE_INPUT)) return FPT_ERR_UNSUPPORTED;
+  if ((flags & FPT_SCALE_INPUT) && !s_in) return FPT_ERR_BAD_ARG;
+  if (post_mode < FPT_POST_NONE || post_mode > FPT_POST_VECTOR) return FPT_ERR_BAD_ARG;
+  if (post_mode == FPT_POST_VECTOR && !post) return FPT_ERR_BAD_ARG;
+  if (!act_qp->symmetric && !wsum) return FPT_ERR_BAD_ARG;
+  if (((uintptr_t)X | (uintptr_t)Wq | (uintptr_t)Y | (uintptr_t)sw | (uintptr_t)wsum) & 15) return FPT_ERR_ALIGNMENT;
+  return FPT_OK;
+}
+
+int linear4_run(cudaStream_t st, const void* X, int M, int K, const uint8_t* Wq, const void* sw, int scale_dtype,
+                const int32_t* wsum, int N, const fpt_qparams* act_qp, int flags, float eps, const float* s_in,
+                int post_mode, const float* post, void* Y, float* s_out, uint8_t* ws) {
+  const size_t gemm_ws = kStatusBytes + gemm_scratch_bytes(M);      // control block + matmul scratch
+  uint8_t* Xq = ws + gemm_ws;
+  float* post_inv = reinterpret_cast<float*>(Xq + up256((size_t)M * K / 2));
+  if (act_quant_launch(st, X, M, K, K, act_qp, flags, eps, nullptr, s_in, Xq, s_out,
+                       post_mode == FPT_POST_INVERSE_OF_PRE ? post_inv : nullptr, nullptr) != cudaSuccess)
+    return FPT_ERR_CUDA;
+  GemmParams P{};
+  P.M = M; P.N = N; P.K = K;
+  P.sw = sw; P.scale_dtype = scale_dtype;
+  P.wsum = act_qp->symmetric ? nullptr : wsum;
+  P.zero_point = act_qp->symmetric ? 0 : act_qp->zero_point;
+  P.a_unsigned = act_qp->symmetric ? 0 : 1;
+  P.act_scale = act_qp->scale;
+  P.post = post_mode == FPT_POST_NONE ? nullptr : post_mode == FPT_POST_VECTOR ? post : post_inv;
+  P.Y = reinterpret_cast<__nv_bfloat16*>(Y);
+  P.status = reinterpret_cast<uint32_t*>(ws);
+  P.scratch = ws + kStatusBytes;
+  return gemm_launch(st, Xq, Wq, P);
+}
+
 }  // namespace fpt
 
 using namespace fpt;
 
-extern "C" int fpt_version(void) { return 100; }
+extern "C" int fpt_version(void) { return 101; }
+
+extern "C" int fpt_set_programmatic_launch(int enabled) {
+  const int old = g_programmatic_launch;
+  g_programmatic_launch = enabled ? 1 : 0;
+  return old;
+}
 
 extern "C" const char* fpt_strerror(int code) {
   switch (code) {
@@ -51,10 +111,11 @@ extern "C" size_t fpt_workspace_bytes(int op, int M, int N, int K) {
       return kStatusBytes + gemm_scratch_bytes(M) + gemm_a8_scratch_bytes(M, N, K);
     case FPT_OP_LINEAR_A8:
       return kStatusBytes + gemm_scratch_bytes(M) + gemm_a8_scratch_bytes(M, N, K) + up256(m * (size_t)K) + up256(m * 4);
-    case FPT_OP_MLP: {   // N = d_ff, K = d
+    case FPT_OP_MLP:
+    case FPT_OP_MLP_HADAMARD: {   // N = d_ff, K = d
       const size_t dff = (size_t)N, d = (size_t)K;
-      return kStatusBytes + gemm_scratch_bytes(M) + up256(m * d / 2) + 2 * up256(m * 4) + up256(m * 2 * dff * 2) +
-             up256(m * dff / 2);
+      return kStatusBytes + gemm_scratch_bytes(M) + up256(m * d / 2) + 2 * up256(m * 4) +
+             up256(mlp_gu_bytes(M, N, op == FPT_OP_MLP_HADAMARD)) + up256(m * dff / 2);
     }
     default:
       return 0;
@@ -134,20 +195,12 @@ extern "C" int fpt_w4a4_linear(void* stream, const void* X, int M, int K, const 
     return fpt_w4a8_gemm(stream, Xq8, Wq, M, N, K, sw, scale_dtype, act_qp->scale, pv8, nullptr, nullptr, Y, nullptr,
                          workspace, gemm_ws8);
   }
-  if (!act_qp->symmetric && !wsum) return FPT_ERR_BAD_ARG;
-  if (((uintptr_t)X | (uintptr_t)Wq | (uintptr_t)Y | (uintptr_t)workspace) & 15) return FPT_ERR_ALIGNMENT;
+  rc = linear4_check(X, Wq, sw, scale_dtype, wsum, Y, act_qp, M, N, K, flags, s_in, post_mode, post);
+  if (rc) return rc;
+  if ((uintptr_t)workspace & 15) return FPT_ERR_ALIGNMENT;
   if (!workspace || workspace_bytes < fpt_workspace_bytes(FPT_OP_LINEAR, M, N, K)) return FPT_ERR_WORKSPACE;
-  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
-  const size_t gemm_ws = kStatusBytes + gemm_scratch_bytes(M);      // control block + matmul scratch
-  uint8_t* Xq = ws + gemm_ws;
-  float* post_inv = reinterpret_cast<float*>(Xq + up256((size_t)M * K / 2));
-  cudaStream_t st = (cudaStream_t)stream;
-  if (act_quant_launch(st, X, M, K, K, act_qp, flags, eps, nullptr, s_in, Xq, s_out,
-                       post_mode == FPT_POST_INVERSE_OF_PRE ? post_inv : nullptr, nullptr) != cudaSuccess)
-    return FPT_ERR_CUDA;
-  const float* pv = post_mode == FPT_POST_NONE ? nullptr : post_mode == FPT_POST_VECTOR ? post : post_inv;
-  return fpt_w4a4_gemm(stream, Xq, Wq, M, N, K, sw, scale_dtype, wsum, act_qp->scale, act_qp->symmetric,
-                       act_qp->zero_point, pv, nullptr, nullptr, Y, nullptr, workspace, gemm_ws);
+  return linear4_run((cudaStream_t)stream, X, M, K, Wq, sw, scale_dtype, wsum, N, act_qp, flags, eps, s_in, post_mode,
+                     post, Y, s_out, reinterpret_cast<uint8_t*>(workspace));
 }
 
 extern "C" int fpt_decoder_mlp(void* stream, const void* X, int M, int d, int d_ff, const uint8_t* Wgu_q,
@@ -167,7 +220,9 @@ extern "C" int fpt_decoder_mlp(void* stream, const void* X, int M, int d, int d_
   if (mid_hadamard && (hadamard_block(d_ff) < 256 || hadamard_block(d_ff) > 4096)) return FPT_ERR_UNSUPPORTED;
   if (((uintptr_t)X | (uintptr_t)Wgu_q | (uintptr_t)Wd_q | (uintptr_t)Y | (uintptr_t)workspace) & 15)
     return FPT_ERR_ALIGNMENT;
-  if (!workspace || workspace_bytes < fpt_workspace_bytes(FPT_OP_MLP, M, d_ff, d)) return FPT_ERR_WORKSPACE;
+  if (!workspace ||
+      workspace_bytes < fpt_workspace_bytes(mid_hadamard ? FPT_OP_MLP_HADAMARD : FPT_OP_MLP, M, d_ff, d))
+    return FPT_ERR_WORKSPACE;
   const size_t m = (size_t)M;
   uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
   const size_t gemm_ws = kStatusBytes + gemm_scratch_bytes(M);      // control block + matmul scratch
@@ -175,14 +230,14 @@ extern "C" int fpt_decoder_mlp(void* stream, const void* X, int M, int d, int d_
   float* sn_ws = reinterpret_cast<float*>(Xq + up256(m * d / 2));
   float* r_ws = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(sn_ws) + up256(m * 4));
   uint8_t* GU = reinterpret_cast<uint8_t*>(r_ws) + up256(m * 4);
-  uint8_t* Mq = GU + up256(m * 2 * (size_t)d_ff * 2);
+  uint8_t* Mq = GU + up256(mlp_gu_bytes(M, d_ff, mid_hadamard != 0));
   float* sn = s_out ? s_out : sn_ws;
   cudaStream_t st = (cudaStream_t)stream;
 
   // X~ = RMSNorm(X) on the grid qp_in; S_n = S_{n-1} * r
   if (act_quant_launch(st, X, M, d, d, qp_in, FPT_RMSNORM, eps, nullptr, s_prev, Xq, sn, nullptr, r_ws) != cudaSuccess)
     return FPT_ERR_CUDA;
-  if (M > 128 && (((uintptr_t)sw_gu | (uintptr_t)sw_d) & 15) == 0) {
+  if (M > 128) {
     // gate || up in one matmul whose epilogue forms m = bf16(silu(g) * u) and quantises m * S_n:
     // the static grid and S_n are known before the matmul starts, so g and u never reach memory
     GemmParams P{};

@@ -36,12 +36,33 @@ __device__ __forceinline__ float load_scale(const void* sw, int scale_dtype, int
                                       : reinterpret_cast<const float*>(sw)[n];
 }
 
+// 32 packed 4-bit codes (16 bytes) -> 32 int8 values code * 16 (8 words): the low nibbles shifted up
+// (out[0..3]: the even-k codes of the 16 bytes), the high nibbles in place (out[4..7]: the odd-k
+// codes).  Both operands of a matmul are widened by this function, so the order of k inside the
+// group does not matter and the accumulator holds 256 * sum.
+__device__ __forceinline__ void widen(const uint4& p, uint32_t* out) {
+  out[0] = (p.x << 4) & 0xF0F0F0F0u;  out[4] = p.x & 0xF0F0F0F0u;
+  out[1] = (p.y << 4) & 0xF0F0F0F0u;  out[5] = p.y & 0xF0F0F0F0u;
+  out[2] = (p.z << 4) & 0xF0F0F0F0u;  out[6] = p.z & 0xF0F0F0F0u;
+  out[3] = (p.w << 4) & 0xF0F0F0F0u;  out[7] = p.w & 0xF0F0F0F0u;
+}
+
 // ----------------------------------------------------------------------------------
 // PTX wrappers
 // ----------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
+
+// Programmatic dependent launch.  A kernel launched with the programmatic-serialisation attribute may
+// start while the kernel before it in the stream is still running; pdl_wait() returns once that
+// kernel has completed and its writes are visible (at once when the launch carried no such
+// attribute), so everything a kernel does before it must not touch memory an earlier kernel may
+// write.  pdl_launch_dependents() lets the NEXT kernel's CTAs be scheduled as soon as every CTA of
+// this grid has called it; the kernels call it right after their own wait, so at most two grids
+// ever overlap.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ uint64_t globaltimer_ns() {
   uint64_t t;
@@ -119,6 +140,13 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const void* tmap, uint
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
       ::"r"(dst), "l"(tmap), "r"(bar), "r"(x), "r"(y)
+      : "memory");
+}
+// 3-D tiled TMA load (no multicast).
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const void* tmap, uint32_t bar, int x, int y, int z) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(tmap), "r"(bar), "r"(x), "r"(y), "r"(z)
       : "memory");
 }
 // 2-D tiled TMA store shared -> global (bulk async group); elements outside the tensor are not written.
@@ -280,6 +308,17 @@ __device__ __forceinline__ void umma_i8_ts_pair(uint32_t d_tmem, uint32_t a_tmem
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::2.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
       ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T over a CTA pair (both operands in shared memory: 128 rows of A and
+// N/2 rows of B in each CTA).
+__device__ __forceinline__ void umma_i8_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                             uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 // The same for a single CTA (A in tensor memory, B in shared memory).

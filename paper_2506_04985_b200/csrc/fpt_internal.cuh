@@ -2,6 +2,7 @@
 #pragma once
 
 #include "fpt_common.cuh"
+#include "fpt_host.cuh"
 
 namespace fpt {
 
@@ -29,6 +30,9 @@ struct GemmParams {
   float mid_inv_delta;         // 1/D of the grid at the down-projection input
   int mid_qmax_minus_z;
   uint32_t mid_flip;
+  int early_weights;           // Wq / sw / wsum are certainly not written by the kernel in front of this one in
+                               // the stream (the library's own quantiser): a kernel may request them before
+                               // its dependency wait
   uint32_t* status;            // control block of the workspace (status word, decode counters)
   void* scratch;               // gemm_scratch_bytes(M) bytes behind the control block (decode partial sums)
 };
@@ -64,5 +68,15 @@ int gemm_decode_small_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* 
 
 // gemm_w4a4_2cta.cu: the CTA-pair kernel (256 x 256 tiles) behind gemm_launch for prefill sizes.
 int gemm_pair_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, const GemmParams& P);
+
+// api.cu: argument checks and body of the 4-bit static linear on a workspace of
+// fpt_workspace_bytes(FPT_OP_LINEAR, M, N, K) bytes whose control block is zero (shared by
+// fpt_w4a4_linear and fpt_w4a4_linear_static).
+int linear4_check(const void* X, const uint8_t* Wq, const void* sw, int scale_dtype, const int32_t* wsum, const void* Y,
+                  const fpt_qparams* act_qp, int M, int N, int K, int flags, const float* s_in, int post_mode,
+                  const float* post);
+int linear4_run(cudaStream_t st, const void* X, int M, int K, const uint8_t* Wq, const void* sw, int scale_dtype,
+                const int32_t* wsum, int N, const fpt_qparams* act_qp, int flags, float eps, const float* s_in,
+                int post_mode, const float* post, void* Y, float* s_out, uint8_t* ws);
 
 }  // namespace fpt

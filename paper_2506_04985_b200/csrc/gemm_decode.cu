@@ -72,13 +72,6 @@ __device__ __forceinline__ long long range_start(const DecodeParams& D, int c, i
   return (D.total * c) / nctas;
 }
 
-__device__ __forceinline__ void widen(const uint4& p, uint32_t* out) {      // 32 codes -> 32 int8 (x16)
-  out[0] = (p.x << 4) & 0xF0F0F0F0u;  out[4] = p.x & 0xF0F0F0F0u;
-  out[1] = (p.y << 4) & 0xF0F0F0F0u;  out[5] = p.y & 0xF0F0F0F0u;
-  out[2] = (p.z << 4) & 0xF0F0F0F0u;  out[6] = p.z & 0xF0F0F0F0u;
-  out[3] = (p.w << 4) & 0xF0F0F0F0u;  out[7] = p.w & 0xF0F0F0F0u;
-}
-
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_w4a4_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                         const DecodeParams D) {
@@ -118,11 +111,6 @@ gemm_w4a4_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     prefetch_tmap(&tmW);
     prefetch_tmap(&tmX);
   }
-  if (threadIdx.x >= kEpiWarp0 * 32 && threadIdx.x < kEpiWarp0 * 32 + kMaxTok) {
-    const int t = threadIdx.x - kEpiWarp0 * 32;
-    c_s[t] = (t < P.M && P.post) ? __fmul_rn(P.act_scale, __ldg(P.post + t)) : P.act_scale;
-    rs_s[t] = (t < P.M && P.res_scale) ? __ldg(P.res_scale + t) : 1.0f;
-  }
   if (warp == 1) {
     tmem_alloc(sbase + L::kMiscOff, kTmemCols);
     tmem_relinquish();
@@ -131,6 +119,8 @@ gemm_w4a4_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = misc[0];
+  pdl_wait();                      // nothing above touched memory another kernel may write
+  pdl_launch_dependents();
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -256,6 +246,15 @@ gemm_w4a4_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     // ------------------------------------------------------------------ epilogue
     const int quad = warp & 3;
     const int npad = D.npad;
+    {
+      // per-token factors of the epilogue, shared by the four epilogue warps
+      const int t = threadIdx.x - kEpiWarp0 * 32;
+      if (t < kMaxTok) {
+        c_s[t] = (t < P.M && P.post) ? __fmul_rn(P.act_scale, __ldg(P.post + t)) : P.act_scale;
+        rs_s[t] = (t < P.M && P.res_scale) ? __ldg(P.res_scale + t) : 1.0f;
+      }
+      named_bar_sync(1, 128);
+    }
     int seg = 0;
     long long g = g_begin;
     while (g < g_end) {
@@ -376,22 +375,6 @@ gemm_w4a4_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
 // ------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
-  return fn;
-}
-
 static bool make_map(CUtensorMap* m, const void* base, int rows, int K, int box_rows, CUtensorMapSwizzle swz) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
@@ -404,16 +387,7 @@ static bool make_map(CUtensorMap* m, const void* base, int rows, int K, int box_
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-static int num_sms() {
-  static int n = 0;
-  if (!n) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    if (n <= 0) n = 1;
-  }
-  return n;
-}
+static int num_sms() { return device_sm_count(); }
 
 }  // namespace decode
 
@@ -427,13 +401,8 @@ size_t gemm_decode_scratch_bytes(int M) {
 // live in the workspace's control block behind the status word.
 int gemm_decode_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, const GemmParams& P, void* scratch) {
   using namespace decode;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(gemm_w4a4_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::kAlloc) !=
-        cudaSuccess)
-      return FPT_ERR_CUDA;
-    attr_set = true;
-  }
+  static PerDeviceInt attr_set;
+  if (!ensure_smem_attr(attr_set, gemm_w4a4_decode_kernel, Smem::kAlloc)) return FPT_ERR_CUDA;
   DecodeParams D;
   D.g = P;
   D.npad = decode_npad(P.M);
@@ -460,8 +429,10 @@ int gemm_decode_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, co
   }
   const long long units = D.whole_tiles ? D.tiles : D.total;
   if (units < ctas) ctas = (int)units;
-  gemm_w4a4_decode_kernel<<<ctas, kThreads, Smem::kAlloc, st>>>(tmW, tmX, D);
-  return cudaGetLastError() == cudaSuccess ? FPT_OK : FPT_ERR_CUDA;
+  return launch_kernel(gemm_w4a4_decode_kernel, dim3(ctas), dim3(kThreads), Smem::kAlloc, st, true, tmW, tmX, D) ==
+                 cudaSuccess
+             ? FPT_OK
+             : FPT_ERR_CUDA;
 }
 
 }  // namespace fpt

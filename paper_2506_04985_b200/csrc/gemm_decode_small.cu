@@ -28,13 +28,6 @@ struct Params {
   int kblocks;                             // 64-byte packed blocks per row: K / 128
 };
 
-__device__ __forceinline__ void widen(const uint4& p, uint32_t* out) {      // 32 codes -> 32 int8 (x16)
-  out[0] = (p.x << 4) & 0xF0F0F0F0u;  out[4] = p.x & 0xF0F0F0F0u;
-  out[1] = (p.y << 4) & 0xF0F0F0F0u;  out[5] = p.y & 0xF0F0F0F0u;
-  out[2] = (p.z << 4) & 0xF0F0F0F0u;  out[6] = p.z & 0xF0F0F0F0u;
-  out[3] = (p.w << 4) & 0xF0F0F0F0u;  out[7] = p.w & 0xF0F0F0F0u;
-}
-
 // C[16x8] += A[16x32] * B[32x8], int8 operands (B signed or unsigned), int32 accumulators.
 template <bool kBUnsigned>
 __device__ __forceinline__ void mma_16x8x32(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -63,6 +56,8 @@ template <int NW, int NT, bool kBUnsigned, bool kA8 = false>
 __global__ void __launch_bounds__(NW * 32, 768 / (NW * 32)) gemm_w4a4_decode_small_kernel(const uint8_t* __restrict__ Xq,
                                                                           const uint8_t* __restrict__ Wq, const Params D) {
   __shared__ int part[NW][kRows][8 * NT];
+  pdl_wait();                      // the activation codes come from the kernel before this one
+  pdl_launch_dependents();
   const GemmParams& P = D.g;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
@@ -178,10 +173,14 @@ __global__ void __launch_bounds__(NW * 32, 768 / (NW * 32)) gemm_w4a4_decode_sma
 template <int NW, int NT>
 static int launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, const Params& D) {
   const int grid = (D.g.N + kRows - 1) / kRows;
-  if (D.g.a_bits == 8) gemm_w4a4_decode_small_kernel<NW, NT, false, true><<<grid, NW * 32, 0, st>>>(Xq, Wq, D);
-  else if (D.g.a_unsigned) gemm_w4a4_decode_small_kernel<NW, NT, true><<<grid, NW * 32, 0, st>>>(Xq, Wq, D);
-  else gemm_w4a4_decode_small_kernel<NW, NT, false><<<grid, NW * 32, 0, st>>>(Xq, Wq, D);
-  return cudaGetLastError() == cudaSuccess ? FPT_OK : FPT_ERR_CUDA;
+  cudaError_t e;
+  if (D.g.a_bits == 8)
+    e = launch_kernel(gemm_w4a4_decode_small_kernel<NW, NT, false, true>, dim3(grid), dim3(NW * 32), 0, st, true, Xq, Wq, D);
+  else if (D.g.a_unsigned)
+    e = launch_kernel(gemm_w4a4_decode_small_kernel<NW, NT, true>, dim3(grid), dim3(NW * 32), 0, st, true, Xq, Wq, D);
+  else
+    e = launch_kernel(gemm_w4a4_decode_small_kernel<NW, NT, false>, dim3(grid), dim3(NW * 32), 0, st, true, Xq, Wq, D);
+  return e == cudaSuccess ? FPT_OK : FPT_ERR_CUDA;
 }
 
 }  // namespace decode_small

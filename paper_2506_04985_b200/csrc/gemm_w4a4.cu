@@ -43,10 +43,10 @@ struct SmemLayout {
 };
 
 __device__ __forceinline__ void expand_nibbles(const uint4& p, uint4& even, uint4& odd) {
-  even.x = (p.x << 4) & 0xF0F0F0F0u;  odd.x = p.x & 0xF0F0F0F0u;
-  even.y = (p.y << 4) & 0xF0F0F0F0u;  odd.y = p.y & 0xF0F0F0F0u;
-  even.z = (p.z << 4) & 0xF0F0F0F0u;  odd.z = p.z & 0xF0F0F0F0u;
-  even.w = (p.w << 4) & 0xF0F0F0F0u;  odd.w = p.w & 0xF0F0F0F0u;
+  uint32_t w[8];
+  widen(p, w);
+  even = make_uint4(w[0], w[1], w[2], w[3]);
+  odd = make_uint4(w[4], w[5], w[6], w[7]);
 }
 
 template <int BN, int NI8, int NPK, int NCONV>
@@ -99,6 +99,8 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = misc[0];
+  pdl_wait();                      // nothing above touched memory another kernel may write
+  pdl_launch_dependents();
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -274,22 +276,6 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 // ------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
-  return fn;
-}
-
 // Tensor map over a packed [rows, K/2]-byte matrix; one box = box_rows rows of one k-block.
 static bool make_packed_map(CUtensorMap* m, const void* base, int rows, int K, int box_rows) {
   EncodeTiledFn fn = encode_fn();
@@ -303,34 +289,24 @@ static bool make_packed_map(CUtensorMap* m, const void* base, int rows, int K, i
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-static int num_sms() {
-  static int n = 0;
-  if (!n) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-  }
-  return n;
-}
+static int num_sms() { return device_sm_count(); }
 
 template <int BN, int NI8, int NPK, int NCONV>
 static int launch_gemm(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, GemmParams P) {
   using L = SmemLayout<BN, NI8, NPK>;
   auto kern = gemm_w4a4_kernel<BN, NI8, NPK, NCONV>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kAlloc) != cudaSuccess)
-      return FPT_ERR_CUDA;
-    attr_set = true;
-  }
+  static PerDeviceInt attr_set;
+  if (!ensure_smem_attr(attr_set, kern, L::kAlloc)) return FPT_ERR_CUDA;
   CUtensorMap tmA, tmB;
   if (!make_packed_map(&tmA, Xq, P.M, P.K, BM) || !make_packed_map(&tmB, Wq, P.N, P.K, BN)) return FPT_ERR_CUDA;
   P.tiles_m = (P.M + BM - 1) / BM;
   P.num_tiles = P.tiles_m * ((P.N + BN - 1) / BN);
   P.kblocks = P.K / BK;
   const int grid = P.num_tiles < num_sms() ? P.num_tiles : num_sms();
-  kern<<<grid, (kFirstConvWarp + NCONV) * 32, L::kAlloc, st>>>(tmA, tmB, P);
-  return cudaGetLastError() == cudaSuccess ? FPT_OK : FPT_ERR_CUDA;
+  return launch_kernel(kern, dim3(grid), dim3((kFirstConvWarp + NCONV) * 32), L::kAlloc, st, true, tmA, tmB, P) ==
+                 cudaSuccess
+             ? FPT_OK
+             : FPT_ERR_CUDA;
 }
 
 int gemm_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, const GemmParams& P) {

@@ -68,26 +68,6 @@ struct Smem {
   static_assert(kAlloc <= 232448, "exceeds the shared memory of one CTA");
 };
 
-__device__ __forceinline__ void widen(const uint4& p, uint32_t* out) {      // 32 codes -> 32 int8 (x16)
-  out[0] = (p.x << 4) & 0xF0F0F0F0u;  out[4] = p.x & 0xF0F0F0F0u;
-  out[1] = (p.y << 4) & 0xF0F0F0F0u;  out[5] = p.y & 0xF0F0F0F0u;
-  out[2] = (p.z << 4) & 0xF0F0F0F0u;  out[6] = p.z & 0xF0F0F0F0u;
-  out[3] = (p.w << 4) & 0xF0F0F0F0u;  out[7] = p.w & 0xF0F0F0F0u;
-}
-
-__device__ __forceinline__ void load_scales8(const void* sw, int scale_dtype, int n, float (&o)[8]) {
-  if (scale_dtype == FPT_DTYPE_F16) {
-    const uint4 h = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const __half*>(sw) + n));
-    const __half2* h2 = reinterpret_cast<const __half2*>(&h);
-#pragma unroll
-    for (int j = 0; j < 4; ++j) { const float2 f = __half22float2(h2[j]); o[2 * j] = f.x; o[2 * j + 1] = f.y; }
-  } else {
-    const float4 a = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(sw) + n));
-    const float4 b = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(sw) + n + 4));
-    o[0] = a.x; o[1] = a.y; o[2] = a.z; o[3] = a.w; o[4] = b.x; o[5] = b.y; o[6] = b.z; o[7] = b.w;
-  }
-}
-
 // kFuse: 0 plain scale-factor epilogue; 1 SwiGLU product + quantiser (codes out); 2 SwiGLU product
 // (bf16 out).  Separate instantiations keep the plain epilogue's register budget free of the others.
 template <int NS, int NPK, int kFuse, bool kA8 = false, int kTN = TN>
@@ -159,6 +139,10 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
   cluster_sync_all();                                  // barriers of both CTAs exist before any remote arrive
   tc_fence_after();
   const uint32_t tmem_base = misc[0];
+  // everything above touched only this CTA pair's own shared and tensor memory; the operands, the
+  // per-token vectors and the outputs may belong to the kernel before this one
+  pdl_wait();
+  pdl_launch_dependents();
 
   // Registers: the epilogue wants the 128 accumulators of its row in registers at once, the other
   // roles need few; the warpgroups trade.  A CTA can only redistribute what it was launched with
@@ -537,22 +521,6 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
 // ------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
-  return fn;
-}
-
 // Tensor map over a packed [rows, K/2]-byte matrix; one box = 128 rows of one k-block (64 bytes each).
 static bool make_map(CUtensorMap* m, const void* base, int rows, int K, CUtensorMapSwizzle swz, int box_rows = HR) {
   EncodeTiledFn fn = encode_fn();
@@ -625,10 +593,9 @@ template <int NS, int NPK, int kFuse, bool kA8 = false, int kTN = TN>
 static int launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, GemmParams P) {
   using L = Smem<NS, NPK, kA8>;
   auto kern = gemm_w4a4_pair_kernel<NS, NPK, kFuse, kA8, kTN>;
-  static int max_pairs = 0;                 // co-resident CTA pairs on this device
-  if (!max_pairs) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kAlloc) != cudaSuccess)
-      return FPT_ERR_CUDA;
+  static PerDeviceInt pairs_cache;          // co-resident CTA pairs on the current device
+  const int max_pairs = pairs_cache.get([&] {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kAlloc) != cudaSuccess) return 0;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2, 1, 1);
     cfg.blockDim = dim3(kThreads, 1, 1);
@@ -640,13 +607,11 @@ static int launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, GemmPar
     int n = 0;
     if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) {
       cudaGetLastError();
-      int dev = 0, sms = 0;
-      cudaGetDevice(&dev);
-      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-      n = sms / 2;
+      n = device_sm_count() / 2;
     }
-    max_pairs = n > 0 ? n : 1;
-  }
+    return n > 0 ? n : 1;
+  });
+  if (max_pairs <= 0) return FPT_ERR_CUDA;
   CUtensorMap tmA, tmB, tmY, tmYt;
   if (!(kA8 ? make_map_i8(&tmA, Xq, P.M, P.K) : make_map(&tmA, Xq, P.M, P.K, CU_TENSOR_MAP_SWIZZLE_64B)) ||
       !make_map(&tmB, Wq, P.N, P.K, CU_TENSOR_MAP_SWIZZLE_NONE, kTN / 2))
@@ -666,22 +631,15 @@ static int launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, GemmPar
   P.num_tiles = P.tiles_m * ((P.N + kTN - 1) / kTN);
   P.kblocks = P.K / BK;
   const int pairs = P.num_tiles < max_pairs ? P.num_tiles : max_pairs;
-  kern<<<2 * pairs, kThreads, L::kAlloc, st>>>(tmA, tmB, tmY, tmYt, tmR, tmRt, P);
-  return cudaGetLastError() == cudaSuccess ? FPT_OK : FPT_ERR_CUDA;
+  return launch_kernel(kern, dim3(2 * pairs), dim3(kThreads), L::kAlloc, st, true, tmA, tmB, tmY, tmYt, tmR, tmRt, P) ==
+                 cudaSuccess
+             ? FPT_OK
+             : FPT_ERR_CUDA;
 }
 
 }  // namespace pair
 
-static int device_pairs() {
-  static int n = 0;
-  if (!n) {
-    int dev = 0, sms = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    n = sms >= 2 ? sms / 2 : 1;
-  }
-  return n;
-}
+static int device_pairs() { const int sms = device_sm_count(); return sms >= 2 ? sms / 2 : 1; }
 
 int gemm_pair_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, const GemmParams& P) {
   if (P.Mq) return pair::launch<4, 5, 1>(st, Xq, Wq, P);

@@ -29,6 +29,8 @@ struct HadQuantParams {
 template <int C>
 __global__ void __launch_bounds__(256) hadamard_quant_kernel(const HadQuantParams P) {
   constexpr int kBlock = 256 * C;
+  pdl_wait();                                    // the products come from the matmul before this kernel
+  pdl_launch_dependents();
   const int lane = threadIdx.x & 31;
   const int groups = P.K / kBlock;
   const long long wid = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
@@ -103,8 +105,7 @@ __global__ void __launch_bounds__(256) hadamard_quant_kernel(const HadQuantParam
 template <int C>
 static cudaError_t launch_had(const HadQuantParams& P, cudaStream_t st) {
   const long long warps = (long long)P.M * (P.K / (256 * C));
-  hadamard_quant_kernel<C><<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(P);
-  return cudaGetLastError();
+  return launch_kernel(hadamard_quant_kernel<C>, dim3((unsigned)((warps + 7) / 8)), dim3(256), 0, st, true, P);
 }
 
 int hadamard_block(int K) { return K & (-K); }

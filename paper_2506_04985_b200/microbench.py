@@ -10,6 +10,7 @@
     python -m paper_2506_04985_b200.microbench gemm_a8   --M 2048 --N 6144 --K 4096       (int8 activation codes)
     python -m paper_2506_04985_b200.microbench linear_dynamic --M 2048 --N 6144 --K 4096 --bits 4
     python -m paper_2506_04985_b200.microbench act_quant_dynamic --M 2048 --K 4096 --bits 4
+    python -m paper_2506_04985_b200.microbench mma_probe                                  (bare tensor-core instruction rates)
 
 Operands are random packed codes / random bf16 values made on the device (timing does
 not depend on the values).  `--sets S` rotates S independent operand sets so that every
@@ -128,7 +129,7 @@ def make_case(kind, M, N, K, sets, dev, f16_scales=False, bits=4):
             sgu = torch.rand((2 * dff,), device=dev).to(sdt) * 0.01 + 0.001
             sd = torch.rand((d,), device=dev).to(sdt) * 0.01 + 0.001
             y = torch.empty((M, d), dtype=torch.bfloat16, device=dev)
-            ws = B.new_workspace(B.OP_MLP, M, dff, d, dev)
+            ws = B.new_workspace(B.OP_MLP_HADAMARD if kind == "mlp_hadamard" else B.OP_MLP, M, dff, d, dev)
             runs.append(lambda x=x, wgu=wgu, sgu=sgu, wd=wd, sd=sd, y=y, ws=ws: B.fpt_decoder_mlp(
                 x, wgu, sgu, wd, sd, qp, qp, 1e-5, want_s_out=False, ws=ws, Y=y, mid_hadamard=kind == "mlp_hadamard"))
         return runs, 6.0 * M * d * dff, 4.0 * M * d + 1.5 * d * dff + 3 * dff * ssz
@@ -169,7 +170,46 @@ def time_case_graph(runs, reps, warmup=3, replays=5):
     return e0.elapsed_time(e1) * 1e3 / (reps * replays)
 
 
+def mma_rate(pair, n, n_acc, a_in_tmem, iters=4096, ctas=None, repeats=5):
+    """Rate of bare 8-bit integer tensor-core instructions (fpt_probe_mma) over all SMs: best of `repeats`
+    launches, CUDA events on the launching stream -> dict with TOP/s and SM cycles per instruction."""
+    dev = torch.device("cuda", torch.cuda.current_device())
+    if ctas is None:
+        ctas = torch.cuda.get_device_properties(dev).multi_processor_count
+        if pair:
+            ctas -= ctas & 1
+    ws = torch.zeros((8192,), dtype=torch.uint8, device=dev)
+    B.fpt_probe_mma(pair, n, n_acc, a_in_tmem, 64, ctas, ws)
+    torch.cuda.synchronize()
+    best, cyc = None, None
+    for _ in range(repeats):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        c = B.fpt_probe_mma(pair, n, n_acc, a_in_tmem, iters, ctas, ws)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        if best is None or ms < best:
+            best, cyc = ms, c
+    assert B.fpt_check_status(ws) == B.OK
+    rows = 256 if pair else 128
+    units = ctas // 2 if pair else ctas
+    ops = 2.0 * rows * n * 32 * 4 * iters * units
+    return {"pair": int(pair), "n": n, "n_acc": n_acc, "a_in_tmem": int(a_in_tmem), "ctas": ctas, "iters": iters,
+            "us": best * 1e3, "tops": ops / (best * 1e-3) / 1e12,
+            "cycles_per_instruction": float(cyc.double().median().item()) / (4 * iters)}
+
+
 def main():
+    if len(__import__("sys").argv) > 1 and __import__("sys").argv[1] == "mma_probe":
+        B.lib()
+        torch.cuda.set_device(0)
+        for pair, n, n_acc, atm in ((1, 256, 1, 1), (1, 256, 1, 0), (1, 240, 1, 1), (0, 256, 1, 1), (0, 256, 1, 0),
+                                    (0, 64, 1, 1), (0, 64, 2, 1), (0, 64, 4, 1), (0, 64, 7, 1), (0, 64, 1, 0), (0, 64, 4, 0),
+                                    (0, 32, 1, 1), (0, 32, 4, 1), (0, 32, 8, 1), (0, 16, 1, 1), (0, 16, 4, 1), (0, 16, 8, 1),
+                                    (0, 128, 1, 1), (0, 128, 2, 1), (1, 64, 1, 1), (1, 64, 4, 1), (1, 128, 1, 1), (1, 128, 2, 1)):
+            print(json.dumps(mma_rate(pair, n, n_acc, atm)))
+        return
     ap = argparse.ArgumentParser()
     ap.add_argument("kind", choices=["gemm", "act_quant", "silu_quant", "hadamard_quant", "linear", "mlp", "mlp_hadamard",
                                      "gemm_a8", "act_quant_dynamic", "linear_dynamic", "attn_proj"])

@@ -54,3 +54,53 @@ def assert_bf16_close(got, want, what=""):
     bad = ~((ulp <= 1) | rel)
     assert not bad.any(), f"{what}: {bad.sum()} of {bad.size} outputs off; worst ulp {ulp.max()}"
     return int((ulp > 0).sum())
+
+
+# ------------------------------------------------------------------------------------------
+# guard bands: every buffer the binding allocates (outputs, codes, per-token vectors, workspaces)
+# sits between two bands of a known pattern, and starts out poisoned, so that a write past either
+# end, or an output the kernel never wrote, is seen even though the comparison itself only covers
+# the valid region
+# ------------------------------------------------------------------------------------------
+GUARD_BYTES = 4096
+GUARD_PATTERN = 0xA5
+POISON = 0xFF               # bf16 / f32: a NaN; int32: -1; codes: 0xFF
+
+
+class GuardedAllocator:
+    def __init__(self):
+        self.live = []          # (raw uint8 tensor, payload bytes)
+
+    def __call__(self, shape, dtype, device):
+        shape = (int(shape),) if isinstance(shape, (int, np.integer)) else tuple(int(s) for s in shape)
+        n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+        padded = (n + 255) // 256 * 256
+        raw = torch.empty((2 * GUARD_BYTES + padded,), dtype=torch.uint8, device=device)
+        raw[:GUARD_BYTES] = GUARD_PATTERN
+        raw[GUARD_BYTES:GUARD_BYTES + n] = POISON
+        raw[GUARD_BYTES + n:] = GUARD_PATTERN
+        self.live.append((raw, n))
+        return raw[GUARD_BYTES:GUARD_BYTES + n].view(dtype).view(shape)
+
+    def check(self, release=True):
+        """Asserts that no band was written; with `release`, forgets the buffers (frees their memory once
+        the test drops its own references)."""
+        for raw, n in self.live:
+            lo = raw[:GUARD_BYTES]
+            hi = raw[GUARD_BYTES + n:]
+            assert bool((lo == GUARD_PATTERN).all()), f"write BEFORE a {n}-byte buffer"
+            assert bool((hi == GUARD_PATTERN).all()), f"write PAST the end of a {n}-byte buffer"
+        if release:
+            self.live = []
+
+
+GUARDS = GuardedAllocator()
+
+
+def guarded_empty(shape, dtype, device=DEV):
+    """A poisoned buffer between guard bands for outputs a test allocates itself."""
+    return GUARDS(shape, dtype, device)
+
+
+def check_guards():
+    GUARDS.check(release=True)

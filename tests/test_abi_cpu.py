@@ -40,8 +40,16 @@ def test_workspace_sizes(B):
     assert B.fpt_workspace_bytes(B.OP_GEMM, 64, 1024, 1024) > B.fpt_workspace_bytes(B.OP_GEMM, 128, 1024, 1024)
     lin = B.fpt_workspace_bytes(B.OP_LINEAR, 2048, 4096, 4096)
     assert lin >= 2048 * 4096 // 2 + 2048 * 4
-    mlp = B.fpt_workspace_bytes(B.OP_MLP, 4096, 14336, 4096)
-    assert mlp >= 4096 * 4096 // 2 + 4096 * 2 * 14336 * 2 + 4096 * 14336 // 2
+    # the MLP block: the 16-bit buffer between the two matmuls is reserved only where a route uses it
+    M, dff, d = 4096, 14336, 4096
+    base = M * d // 2 + M * dff // 2                   # codes at the block input and at the down-projection input
+    fused = B.fpt_workspace_bytes(B.OP_MLP, M, dff, d)
+    assert base <= fused < base + (1 << 20), "fused route (more than 128 tokens): no gate||up buffer"
+    had = B.fpt_workspace_bytes(B.OP_MLP_HADAMARD, M, dff, d)
+    assert base + M * dff * 2 <= had < base + M * dff * 2 + (1 << 20), "with the transform: the bf16 products"
+    for op in (B.OP_MLP, B.OP_MLP_HADAMARD):
+        small = B.fpt_workspace_bytes(op, 64, dff, d)
+        assert small >= 64 * d // 2 + 64 * dff // 2 + 64 * 2 * dff * 2, "unfused route: gate||up in bf16"
     assert B.fpt_workspace_bytes(99, 1, 1, 1) == 0
     assert B.fpt_workspace_bytes(B.OP_GEMM, 0, 8, 128) == 0
 

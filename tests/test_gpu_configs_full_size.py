@@ -7,8 +7,9 @@ import pytest
 import torch
 
 from oracle import quantizers as OQ, linear as OL
+from oracle.hadamard import block_hadamard_f32
 from paper_2506_04985_b200 import binding as B, synth
-from helpers import dev, host, oqp, bf16_host, assert_bf16_close
+from helpers import dev, host, oqp, bf16_host, assert_bf16_close, check_guards
 
 pytestmark = pytest.mark.gpu
 
@@ -16,6 +17,26 @@ pytestmark = pytest.mark.gpu
 def _rows(M, n=10):
     base = [0, 1, 127, 128, 255, 256, 257, M // 2 - 1, M // 2, M - 257, M - 256, M - 129, M - 2, M - 1]
     return np.unique(np.clip(np.array(base), 0, M - 1))
+
+
+def _rows_sample(M, n=256):
+    """At least n rows: the first and last rows of every 256-row tile's two 128-row halves near the ends and
+    the middle of the matrix, plus seeded random rows."""
+    tiles = sorted({0, 1, M // 512, M // 256 - 2, M // 256 - 1} & set(range(M // 256)))
+    edge = [t * 256 + o for t in tiles for o in (0, 1, 127, 128, 254, 255)]
+    rng = np.random.default_rng(M)
+    rows = np.unique(np.concatenate([np.array(edge), _rows(M), rng.choice(M, size=n, replace=False)]))
+    return rows[rows < M]
+
+
+_WQ_CACHE = {}
+
+
+def _oracle_weights(name, w):
+    """Oracle-side weight codes of a seeded matrix (the same matrix serves every token count)."""
+    if name not in _WQ_CACHE:
+        _WQ_CACHE[name] = OQ.quantize_weights(synth.f32(w))
+    return _WQ_CACHE[name]
 
 
 def test_config3_mlp_block_4096_tokens_sampled():
@@ -47,12 +68,13 @@ def test_config3_mlp_block_4096_tokens_sampled():
     assert assert_bf16_close(bf16_host(Y)[rows], ref["y"], "cfg3 Y") == 0
 
 
-@pytest.mark.parametrize("tokens", [512, 2048])
+@pytest.mark.parametrize("tokens", [512, 2048, 8192])
 def test_config5_70b_class_linears_sampled(tokens):
     """hidden 8192, MLP 28672, 8 kv heads x 128: fused QKV (10240), O, gate||up as two linears, down;
-    weights with outlier rows, activations with outlier channels x60."""
+    weights with outlier rows, activations with outlier channels x60.  At 2048 and 8192 tokens the
+    oracle runs on a seeded sample of at least 256 token rows (tile edges included), all columns."""
     M, h, d_ff = tokens, 8192, 28672
-    rows = _rows(M)
+    rows = _rows(M) if tokens == 512 else _rows_sample(M)
 
     def run(K, N, name, flags, scale):
         x = synth.activations(M, K, 0, f"cfg5/x{name}", law="student_t3", outlier_frac=0.005, outlier_gain=60.0)
@@ -60,7 +82,7 @@ def test_config5_70b_class_linears_sampled(tokens):
         s_in = synth.per_token_scale(M, 0, f"cfg5/s{name}")
         qp = B.QParams(4, True, scale, 0)
         wq, sw, _ = B.fpt_quantize_weights(dev(w))
-        cw, d, _ = OQ.quantize_weights(synth.f32(w))
+        cw, d, _ = _oracle_weights(name, w)
         assert np.array_equal(host(sw), d)
         ws = B.new_workspace(B.OP_LINEAR, M, N, K)
         Y, s_out = B.fpt_w4a4_linear(dev(x), wq, sw, qp, flags, 1e-5, s_in=dev(s_in), ws=ws)
@@ -70,11 +92,42 @@ def test_config5_70b_class_linears_sampled(tokens):
         assert len(np.unique(ref["codes"])) >= 8
         assert np.array_equal(host(s_out)[rows], ref["s_out"])
         assert assert_bf16_close(bf16_host(Y)[rows], ref["y"], f"cfg5 {name}") == 0
-        del x, w
+        del x, w, Y, s_out, ws, wq, sw
+        check_guards()                     # also lets go of this linear's buffers before the next one
         torch.cuda.empty_cache()
 
     run(h, 10240, "qkv", B.RMSNORM, 0.45)
     run(h, h, "o", B.SCALE_INPUT, 2.5)
-    if tokens == 512:                      # the wide MLP matrices once: their oracle side is the slow part
+    if tokens != 2048:                     # the wide MLP matrices at the smallest and the largest token count
         run(h, d_ff, "gate", B.RMSNORM, 0.45)
         run(d_ff, h, "down", B.SCALE_INPUT, 2.5)
+
+
+def test_mlp_block_with_online_hadamard_4096_tokens_sampled():
+    """The MLP block of configuration 3 with the block Hadamard at the down-projection input
+    (14336 = 7 x 2048; its inverse folded into the down weights is the caller's business: here the
+    down matrix is simply a seeded matrix), sampled rows against the oracle."""
+    M, d, d_ff = 4096, 4096, 14336
+    x = synth.activations(M, d, 1, "cfg3h/x", law="student_t3", outlier_frac=0.005, outlier_gain=50.0)
+    wg = synth.weights(d_ff, d, 0.02, 1, "cfg3h/wg")
+    wu = synth.weights(d_ff, d, 0.02, 1, "cfg3h/wu")
+    wd = synth.weights(d, d_ff, 0.02, 1, "cfg3h/wd")
+    rows = _rows(M)
+    xf = synth.f32(x)[rows]
+    (cg, sg, _), (cu, su, _), (cd, sd, _) = (OQ.quantize_weights(synth.f32(w)) for w in (wg, wu, wd))
+    r = OQ.rms_reciprocal(xf, 1e-5)
+    qp_in = B.QParams(4, True, float(OQ.calibrate_static_scale(xf * r[:, None], OQ.QParams())), 0)
+    pre = OL.decoder_mlp(xf, cg, sg, cu, su, cd, sd, oqp(qp_in), OQ.QParams(4, True, 1.0), 1e-5)
+    hm = block_hadamard_f32(pre["m"]) * pre["s_out"][:, None]
+    qp_mid = B.QParams(4, True, float(OQ.calibrate_static_scale(hm, OQ.QParams())), 0)
+    gq, gs, _ = B.fpt_quantize_weights(dev(wg))
+    uq, us, _ = B.fpt_quantize_weights(dev(wu))
+    dq, ds, _ = B.fpt_quantize_weights(dev(wd))
+    wgu, swgu = B.fpt_interleave_gate_up(gq, uq, gs, us)
+    ws = B.new_workspace(B.OP_MLP_HADAMARD, M, d_ff, d)
+    Y, s_out = B.fpt_decoder_mlp(dev(x), wgu, swgu, dq, ds, qp_in, qp_mid, 1e-5, None, True, ws=ws, mid_hadamard=True)
+    assert B.fpt_check_status(ws) == B.OK
+    ref = OL.decoder_mlp(xf, cg, sg, cu, su, cd, sd, oqp(qp_in), oqp(qp_mid), 1e-5, None, True, hadamard=True)
+    assert np.array_equal(host(s_out)[rows], ref["s_out"])
+    assert len(np.unique(ref["mq"])) >= 8
+    assert assert_bf16_close(bf16_host(Y)[rows], ref["y"], "cfg3 + Hadamard Y") == 0
