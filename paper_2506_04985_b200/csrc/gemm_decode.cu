@@ -15,9 +15,12 @@
 // quadrant) adds the slots up -- integer addition, so the result does not depend on the order
 // -- and runs the epilogue.  No CTA ever waits for another.
 //
-// Roles (16 warps): warp 0 TMA producer, warp 1 MMA issuer and tensor-memory owner, warps 2-3
-// token converters, warps 4-11 weight converters (two groups taking alternate k-blocks),
-// warps 12-15 epilogue.
+// Roles (24 warps): warp 0 TMA producer, warp 1 MMA issuer and tensor-memory owner, warps 2-3
+// token converters, warps 4-19 weight converters (four groups of four warps, each group taking every
+// fourth k-block: the chain load -> widen -> tcgen05.st -> wait -> arrive is long, and one
+// tcgen05.mma of 128 rows x 32 codes takes about 100 cycles whatever its width, so four k-blocks in
+// conversion are what keeps the tensor core's queue from running dry), warps 20-23 epilogue.
+// Registers are traded between the warpgroups (setmaxnreg): the epilogue holds 64 accumulators per thread.
 #include <cuda.h>
 
 #include "fpt_internal.cuh"
@@ -29,14 +32,21 @@ constexpr int HR = 128;                    // weight rows per tile
 constexpr int BK = 256;                    // codes per k-block: 128 packed bytes per row, one full cache line
 constexpr int PK_ROW = BK / 2;
 constexpr int I8_ROW = 128;                // the widened token tile is two 128-byte-swizzled halves of 128 codes
-constexpr int NS = 4;                      // widened stages: 4 x 64 tensor-memory columns + 4 token tiles
-constexpr int NPK = 6;                     // packed stages in flight from TMA
+constexpr int NS = 6;                      // widened stages: 6 x 64 tensor-memory columns + 6 token tiles
+constexpr int NPK = 4;                     // packed stages in flight from TMA
+constexpr int kGroups = 4;                 // weight-converter groups
 constexpr int kMaxTok = 64;
 constexpr int kAccCols = 64;               // per accumulator buffer (two of them)
 constexpr int kAStage0 = 2 * kAccCols;
 constexpr int kTmemCols = 512;
-constexpr int kThreads = 512;
-constexpr int kConvBWarp0 = 2, kConvAWarp0 = 4, kEpiWarp0 = 12;
+constexpr int kConvBWarp0 = 2, kConvAWarp0 = 4, kEpiWarp0 = kConvAWarp0 + 4 * kGroups;
+constexpr int kThreads = 32 * (kEpiWarp0 + 4);
+// registers per thread after the trade: warps 0-3, each converter group, the epilogue group
+constexpr int kRegsLaunch = (65536 / kThreads) / 8 * 8, kRegsCtl = 64, kRegsConv = 64, kRegsEpi = 152;
+static_assert(kThreads * kRegsLaunch <= 65536, "launch allocation exceeds the register file");
+static_assert(128 * (kRegsCtl + kGroups * kRegsConv + kRegsEpi) <= kThreads * kRegsLaunch,
+              "the warpgroups ask for more registers than the CTA was launched with: setmaxnreg.inc would never return");
+static_assert(2 * kAccCols + NS * (BK / 4) <= kTmemCols, "operand stages must fit beside the two accumulators");
 
 struct Smem {
   static constexpr int kB8Half = kMaxTok * I8_ROW;                  // 8 KB: 64 token rows x 128 codes as int8
@@ -61,6 +71,7 @@ struct DecodeParams {
   int tiles;               // N / 128 rounded up
   int kblocks;             // K / 256 rounded up (a half block at the end reads zeros past the row)
   long long total;         // tiles * kblocks
+  int per, rem;            // total = per * CTAs + rem: CTA c takes per k-blocks, the first rem CTAs one more
   int whole_tiles;         // 1: ranges end on tile boundaries (no partial sums, no counters)
   int32_t* slots;          // [gridDim.x][2][npad][128] raw int32 partial sums
   uint32_t* counters;      // [tiles][4], zero between launches
@@ -68,8 +79,8 @@ struct DecodeParams {
 
 // First weight k-block (global index) of CTA c's range.
 __device__ __forceinline__ long long range_start(const DecodeParams& D, int c, int nctas) {
-  if (D.whole_tiles) return (long long)D.kblocks * (((long long)D.tiles * c) / nctas);
-  return (D.total * c) / nctas;
+  if (D.whole_tiles) return (long long)D.kblocks * (long long)((unsigned)(D.tiles * c) / (unsigned)nctas);
+  return (long long)c * D.per + (c < D.rem ? c : D.rem);          // no division: this runs inside the epilogue
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -122,6 +133,9 @@ gemm_w4a4_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
   pdl_wait();                      // nothing above touched memory another kernel may write
   pdl_launch_dependents();
 
+  // Registers: the epilogue wants the 64 accumulators of its row in registers at once, the other roles
+  // need few; the warpgroups trade (see the static_assert above: the requests are covered).
+  if (warp < kConvAWarp0) reg_dec<kRegsCtl>();
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -215,27 +229,35 @@ gemm_w4a4_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     }
   } else if (warp < kEpiWarp0) {
     // ------------------------------------------------------------------ weight converters -> tensor memory
+    reg_dec<kRegsConv>();
     const int quad = warp & 3;                           // TMEM lanes this warp may touch
-    const int grp = (warp - kConvAWarp0) >> 2;           // takes the k-blocks whose running index has this parity
+    const int grp = (warp - kConvAWarp0) >> 2;           // takes the k-blocks whose running index is grp modulo kGroups
     const int r = quad * 32 + lane;
     const uint32_t swz = (uint32_t)(r & 7);              // SWIZZLE_128B of the packed weight tile
-    long long kc = grp;                                  // running k-block index of this CTA
-    for (long long g = g_begin + grp; g < g_end; g += 2, kc += 2) {
-      const int ps = (int)(kc % NPK); const uint32_t pph = (uint32_t)((kc / NPK) & 1);
-      const int s = (int)(kc % NS);   const uint32_t ph = (uint32_t)((kc / NS) & 1);
+    const int n_local = (int)(g_end - g_begin);          // k-blocks of this CTA
+    for (int kc = grp; kc < n_local; kc += kGroups) {    // kc: running k-block index of this CTA
+      const int ps = kc % NPK; const uint32_t pph = (uint32_t)((kc / NPK) & 1);
+      const int s = kc % NS;   const uint32_t ph = (uint32_t)((kc / NS) & 1);
       if (!mbar_wait(pk_full(ps), pph, abort_flag, P.status, 5)) break;
       const uint8_t* src = smem + L::kPkWOff + ps * L::kPkW + r * PK_ROW;
-      uint4 c[8];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) c[j] = *reinterpret_cast<const uint4*>(src + (((uint32_t)j ^ swz) << 4));
-      uint32_t v[64];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) widen(c[j], v + 8 * j);
-      if (!mbar_wait(op_empty(s), ph ^ 1u, abort_flag, P.status, 6)) break;
-      tc_fence_after();
       const uint32_t a_tmem = tmem_base + ((uint32_t)(quad * 32) << 16) + kAStage0 + s * (BK / 4);
-      tmem_st_32x32(a_tmem, v);
-      tmem_st_32x32(a_tmem + 32, v + 32);
+      bool ok = true;
+      // the row's 256 codes in two halves of 128 (32 tensor-memory columns each): fewer live registers
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        uint4 c[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) c[j] = *reinterpret_cast<const uint4*>(src + (((uint32_t)(4 * h + j) ^ swz) << 4));
+        uint32_t v[32];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) widen(c[j], v + 8 * j);
+        if (h == 0) {
+          if (!mbar_wait(op_empty(s), ph ^ 1u, abort_flag, P.status, 6)) { ok = false; break; }
+          tc_fence_after();
+        }
+        tmem_st_32x32(a_tmem + 32 * h, v);
+      }
+      if (!ok) break;
       tmem_wait_st();
       tc_fence_before();
       fence_proxy_async_smem();      // reads of the packed tile (consumed above) before the TMA write that re-fills it
@@ -244,6 +266,7 @@ gemm_w4a4_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     }
   } else {
     // ------------------------------------------------------------------ epilogue
+    reg_inc<kRegsEpi>();
     const int quad = warp & 3;
     const int npad = D.npad;
     {
@@ -310,27 +333,20 @@ gemm_w4a4_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
           __threadfence();
 #pragma unroll
           for (int t = 0; t < kMaxTok; ++t) v[t] = 0;
-          if (npad == 16) {
-            // few values per contributor: keep the loads of four contributors in flight together
-            for (int c = c_first; c <= c_last; c += 4) {
-              uint32_t w[4][16];
+          // (sixteen loads in flight per batch: the four epilogue warps are alone on the SM by now, so
+          // nothing else hides the latency of a dependent chain)
+          for (int c = c_first; c <= c_last; ++c) {
+            const int cs = (range_start(D, c, nctas) >= t_begin) ? 0 : 1;
+            const int32_t* src = D.slots + ((size_t)(c * 2 + cs) * npad) * HR + quad * 32 + lane;
 #pragma unroll
-              for (int u = 0; u < 4; ++u) {
-                const int cc = c + u <= c_last ? c + u : c_last;
-                const int cs = (range_start(D, cc, nctas) >= t_begin) ? 0 : 1;
-                const int32_t* src = D.slots + ((size_t)(cc * 2 + cs) * npad) * HR + quad * 32 + lane;
+            for (int t0 = 0; t0 < kMaxTok; t0 += 16) {
+              if (t0 < npad) {
+                uint32_t w[16];
 #pragma unroll
-                for (int t = 0; t < 16; ++t) w[u][t] = (c + u <= c_last) ? (uint32_t)__ldcg(src + (size_t)t * HR) : 0u;
+                for (int t = 0; t < 16; ++t) w[t] = (uint32_t)__ldcg(src + (size_t)(t0 + t) * HR);
+#pragma unroll
+                for (int t = 0; t < 16; ++t) v[t0 + t] += w[t];
               }
-#pragma unroll
-              for (int t = 0; t < 16; ++t) v[t] += (w[0][t] + w[1][t]) + (w[2][t] + w[3][t]);
-            }
-          } else {
-            for (int c = c_first; c <= c_last; ++c) {
-              const int cs = (range_start(D, c, nctas) >= t_begin) ? 0 : 1;
-              const int32_t* src = D.slots + ((size_t)(c * 2 + cs) * npad) * HR + quad * 32 + lane;
-#pragma unroll
-              for (int t = 0; t < kMaxTok; ++t) if (t < npad) v[t] += (uint32_t)__ldcg(src + (size_t)t * HR);
             }
           }
           if (lane == 0) D.counters[tile * 4 + quad] = 0;      // ready for the next launch
@@ -344,15 +360,38 @@ gemm_w4a4_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         int32_t* const acc_out = P.acc_out ? P.acc_out + n : nullptr;
         __nv_bfloat16* const yp = P.Y ? P.Y + n : nullptr;
         const __nv_bfloat16* const resp = P.residual ? P.residual + n : nullptr;
+        if (yp && !acc_out && !resp) {
+          // the usual case, straight-line: sixteen outputs computed, then sixteen stores
 #pragma unroll
-        for (int t = 0; t < kMaxTok; ++t) {
-          if (t < m_tok) {
-            const int a = (((int)v[t]) >> 8) - zw;
-            if (acc_out) acc_out[(size_t)t * ldy] = a;
-            if (yp) {
-              float y = __fmul_rn(__fmul_rn((float)a, swn), c_s[t]);
-              if (resp) y = __fadd_rn(y, __fmul_rn(__bfloat162float(resp[(size_t)t * ldy]), rs_s[t]));
-              yp[(size_t)t * ldy] = __float2bfloat16_rn(y);
+          for (int t0 = 0; t0 < kMaxTok; t0 += 16) {
+            if (t0 < m_tok) {
+              __nv_bfloat16 y[16];
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                const float4 c4 = *reinterpret_cast<const float4*>(c_s + t0 + 4 * q);
+                const float cc[4] = {c4.x, c4.y, c4.z, c4.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  const int a = (((int)v[t0 + 4 * q + j]) >> 8) - zw;
+                  y[4 * q + j] = __float2bfloat16_rn(__fmul_rn(__fmul_rn((float)a, swn), cc[j]));
+                }
+              }
+              __nv_bfloat16* o = yp + (size_t)t0 * ldy;
+#pragma unroll
+              for (int t = 0; t < 16; ++t) if (t0 + t < m_tok) o[(size_t)t * ldy] = y[t];
+            }
+          }
+        } else {
+#pragma unroll
+          for (int t = 0; t < kMaxTok; ++t) {
+            if (t < m_tok) {
+              const int a = (((int)v[t]) >> 8) - zw;
+              if (acc_out) acc_out[(size_t)t * ldy] = a;
+              if (yp) {
+                float y = __fmul_rn(__fmul_rn((float)a, swn), c_s[t]);
+                if (resp) y = __fadd_rn(y, __fmul_rn(__bfloat162float(resp[(size_t)t * ldy]), rs_s[t]));
+                yp[(size_t)t * ldy] = __float2bfloat16_rn(y);
+              }
             }
           }
         }
@@ -426,9 +465,13 @@ int gemm_decode_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, co
     const int max_split = D.kblocks / 2 > 0 ? D.kblocks / 2 : 1;      // at least 2 k-blocks (512 codes) per range
     if (split > max_split) split = max_split;
     ctas = D.tiles * split;
+    // (112 tiles stay on 112 SMs: cutting them into 148 equal ranges was measured slower, 19.4 against
+    // 14.4 us at 64 tokens -- the partial sums of a split tile are 32 KB per range)
   }
   const long long units = D.whole_tiles ? D.tiles : D.total;
   if (units < ctas) ctas = (int)units;
+  D.per = (int)(D.total / ctas);
+  D.rem = (int)(D.total % ctas);
   return launch_kernel(gemm_w4a4_decode_kernel, dim3(ctas), dim3(kThreads), Smem::kAlloc, st, true, tmW, tmX, D) ==
                  cudaSuccess
              ? FPT_OK
