@@ -31,6 +31,12 @@ __device__ __forceinline__ uint32_t f32_to_bf16_bits(float x) {
   return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(x));
 }
 
+// Two float32 values -> two bf16 (round to nearest even each) in one word, lo in bits 0..15.
+__device__ __forceinline__ uint32_t f32x2_to_bf16x2_bits(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+
 __device__ __forceinline__ float load_scale(const void* sw, int scale_dtype, int n) {
   return scale_dtype == FPT_DTYPE_F16 ? __half2float(reinterpret_cast<const __half*>(sw)[n])
                                       : reinterpret_cast<const float*>(sw)[n];
