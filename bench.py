@@ -33,7 +33,7 @@ EPS = 1e-5
 NSETS = 4
 # dram__bytes_read.sum + dram__bytes_write.sum of one fused-QKV matmul launch, from the ncu capture
 # summarised in profiles/gemm_w4a4_pair_2048x6144x4096.md (set to None when the kernel changes)
-GEMM_QKV_DRAM_BYTES = 16.93e6
+GEMM_QKV_DRAM_BYTES = 16.98e6
 METRIC = "W4A4 linear TOPS (prefill, Llama-3-8B-shaped attention projections, 2048 tokens)"
 
 
@@ -453,13 +453,23 @@ def run_gpu(args):
         torch.cuda.empty_cache()
 
         def measure(kind, M, N, K, reps, f16=False):
-            nsets = max(2, min(8, int(300e6 / max(1.0, N * K / 2))))
+            nsets = max(2, min(8, int(300e6 / max(1.0, N * K / 2 + M * K / 2 + 2.0 * M * N))))
             runs, ops, nbytes = MB.make_case(kind, M, N, K, nsets, dev, f16)
             us = MB.time_case_graph(runs, reps)
             del runs
             torch.cuda.empty_cache()
             return us, ops, nbytes
 
+        # configs[0]: one small linear (quantise + matmul), and the separate projections of configs[1]
+        us, ops, _ = measure("linear", 128, 1024, 1024, 50)
+        other["configs[0] single linear 128x1024x1024 (quantise + matmul)"] = {"us": us, "TOP/s": ops / us / 1e6}
+        sep = {}
+        for name, n in (("Q", 4096), ("K", 1024), ("V", 1024), ("O", 4096), ("QKV fused", 6144)):
+            us, ops, _ = measure("gemm", M_TOK, n, HID, 50)
+            sep[name] = {"us": us, "TOP/s": ops / us / 1e6, "frac_of_int8_peak": ops / us / 1e6 / int8_peak}
+        us, _, nbytes = measure("act_quant", M_TOK, 0, HID, 50)
+        sep["act_quant 2048x4096"] = {"us": us, "GB/s": nbytes / us / 1e3, "frac_of_hbm_peak": nbytes / us / 1e3 / peaks["hbm_gbs"]}
+        other["configs[1] projections one by one (matmul + scale factors only)"] = sep
         us, ops, _ = measure("mlp", 4096, D_FF, HID, 10)
         other["configs[2] SwiGLU MLP block, 4096 tokens (4 kernels)"] = {
             "us": us, "TOP/s": ops / us / 1e6, "frac_of_int8_peak": ops / us / 1e6 / int8_peak}

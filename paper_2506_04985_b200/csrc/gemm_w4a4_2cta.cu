@@ -43,6 +43,13 @@ constexpr int kAStageCols = BK / 4;        // 32 columns hold 128 int8 per lane
 constexpr int kTmemCols = 512;
 constexpr int kThreads = 640;
 constexpr int kConvAWarp0 = 4, kConvBWarp0 = 8, kEpiWarp0 = 12, kEpiWarps = 8;
+// Registers per thread: what the CTA is launched with, and what the roles trade it into (warps 0-3,
+// activation converters, weight converters, epilogue).  A CTA can only redistribute what it owns: an
+// increase that the decreases do not cover would never return, so the sum is checked here.
+constexpr int kRegsLaunch = 96, kRegsCtl = 48, kRegsConvA = 56, kRegsConvB = 56, kRegsEpi = 152;
+static_assert(kThreads * kRegsLaunch <= 65536, "launch allocation exceeds the register file");
+static_assert(128 * (kRegsCtl + kRegsConvA + kRegsConvB) + 32 * kEpiWarps * kRegsEpi <= kThreads * kRegsLaunch,
+              "the warpgroups ask for more registers than the CTA was launched with: setmaxnreg.inc would never return");
 
 // NS: stages of widened operands (int8 weight tile in shared memory + activation columns in
 // tensor memory); NPK: stages of packed tiles in flight from TMA.
@@ -150,7 +157,7 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
   // epilogue groups is always met once the three other groups have given theirs back.  Each role
   // branch starts with its own re-allocation (the compiler budgets registers per branch).
   if (warp < kConvAWarp0) {
-    reg_dec<48>();
+    reg_dec<kRegsCtl>();
     if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -205,7 +212,7 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     }
   } else if (warp < kConvBWarp0) {
     // ------------------------------------------------------------------ activation converters -> tensor memory
-    reg_dec<56>();
+    reg_dec<kRegsConvA>();
     const int quad = warp - kConvAWarp0;                 // == warp % 4: the TMEM lanes this warp may touch
     const int r = quad * 32 + lane;                      // row of the CTA's 128
     const uint32_t swz = (uint32_t)((r >> 1) & 3);       // SWIZZLE_64B: 16-byte chunk index ^= (row / 2) % 4
@@ -274,7 +281,7 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     }
   } else if (warp < kEpiWarp0) {
     // ------------------------------------------------------------------ weight converters -> shared int8 tile
-    reg_dec<56>();
+    reg_dec<kRegsConvB>();
     const int ctid = threadIdx.x - kConvBWarp0 * 32;     // 0..127
     const uint32_t op_full_leader = map_to_cta(op_full(0), 0);
     int ps = 0, s = 0; uint32_t pph = 0, ph = 0;
@@ -311,7 +318,7 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     }
   } else {
     // ------------------------------------------------------------------ epilogue
-    reg_inc<152>();
+    reg_inc<kRegsEpi>();
     const int quad = warp & 3;                           // TMEM lane quadrant this warp may read
     const int half = (warp - kEpiWarp0) >> 2;            // which 128 of the 256 columns
     const int etid = (warp - kEpiWarp0) * 32 + lane;     // 0..255: the tile column whose scale this thread fetches
