@@ -14,12 +14,20 @@
 // a scratch slot; the last CTA to arrive at a tile (an atomic counter per tile and lane
 // quadrant) adds the slots up -- integer addition, so the result does not depend on the order
 // -- and runs the epilogue.  No CTA ever waits for another.
+// Where every tile is cut into the same 2, 4 or 8 ranges (few tiles, long rows), the CTAs of a tile are
+// launched as one thread-block cluster instead: each leaves its partial sums in its OWN shared
+// memory, the cluster synchronises once, and every CTA then adds up and finishes its share of the
+// tokens by reading the others' shared memory directly -- no trip through L2, no atomics, and the
+// final epilogue is spread over all CTAs of the tile.  (A cluster barrier does wait for the peers,
+// but they are co-scheduled by construction and all reach it.)
 //
-// Roles (24 warps): warp 0 TMA producer, warp 1 MMA issuer and tensor-memory owner, warps 2-3
-// token converters, warps 4-19 weight converters (four groups of four warps, each group taking every
-// fourth k-block: the chain load -> widen -> tcgen05.st -> wait -> arrive is long, and one
-// tcgen05.mma of 128 rows x 32 codes takes about 100 cycles whatever its width, so four k-blocks in
-// conversion are what keeps the tensor core's queue from running dry), warps 20-23 epilogue.
+// Roles (24 warps): warp 0 TMA producer, warp 1 MMA issuer and tensor-memory owner (warps 2-3 idle),
+// warps 4-7 token converters (with 64 tokens their tile is half as many bytes as the weights': two
+// warps were the slowest stage of the pipeline), warps 8-19 weight converters (three groups of four
+// warps, each group taking every third k-block: the chain load -> widen -> tcgen05.st -> wait -> arrive
+// is long, and one tcgen05.mma of 128 rows x 32 codes takes about 100 cycles whatever its width, so
+// several k-blocks in conversion are what keeps the tensor core's queue from running dry),
+// warps 20-23 epilogue.
 // Registers are traded between the warpgroups (setmaxnreg): the epilogue holds 64 accumulators per thread.
 #include <cuda.h>
 
@@ -34,17 +42,19 @@ constexpr int PK_ROW = BK / 2;
 constexpr int I8_ROW = 128;                // the widened token tile is two 128-byte-swizzled halves of 128 codes
 constexpr int NS = 6;                      // widened stages: 6 x 64 tensor-memory columns + 6 token tiles
 constexpr int NPK = 4;                     // packed stages in flight from TMA
-constexpr int kGroups = 4;                 // weight-converter groups
+constexpr int kGroups = 3;                 // weight-converter groups
+constexpr int kTokWarps = 4;               // token-converter warps
 constexpr int kMaxTok = 64;
 constexpr int kAccCols = 64;               // per accumulator buffer (two of them)
 constexpr int kAStage0 = 2 * kAccCols;
 constexpr int kTmemCols = 512;
-constexpr int kConvBWarp0 = 2, kConvAWarp0 = 4, kEpiWarp0 = kConvAWarp0 + 4 * kGroups;
+constexpr int kConvBWarp0 = 4, kConvAWarp0 = kConvBWarp0 + kTokWarps, kEpiWarp0 = kConvAWarp0 + 4 * kGroups;
 constexpr int kThreads = 32 * (kEpiWarp0 + 4);
 // registers per thread after the trade: warps 0-3, each converter group, the epilogue group
-constexpr int kRegsLaunch = (65536 / kThreads) / 8 * 8, kRegsCtl = 64, kRegsConv = 64, kRegsEpi = 152;
+constexpr int kRegsLaunch = (65536 / kThreads) / 8 * 8, kRegsCtl = 64, kRegsTok = 64, kRegsConv = 64, kRegsEpi = 152;
+static_assert(kTokWarps == 4, "the token converters are one warpgroup");
 static_assert(kThreads * kRegsLaunch <= 65536, "launch allocation exceeds the register file");
-static_assert(128 * (kRegsCtl + kGroups * kRegsConv + kRegsEpi) <= kThreads * kRegsLaunch,
+static_assert(128 * (kRegsCtl + kRegsTok + kGroups * kRegsConv + kRegsEpi) <= kThreads * kRegsLaunch,
               "the warpgroups ask for more registers than the CTA was launched with: setmaxnreg.inc would never return");
 static_assert(2 * kAccCols + NS * (BK / 4) <= kTmemCols, "operand stages must fit beside the two accumulators");
 
@@ -73,6 +83,8 @@ struct DecodeParams {
   long long total;         // tiles * kblocks
   int per, rem;            // total = per * CTAs + rem: CTA c takes per k-blocks, the first rem CTAs one more
   int whole_tiles;         // 1: ranges end on tile boundaries (no partial sums, no counters)
+  int cluster;             // > 1: every tile is cut into this many equal ranges and the CTAs of a range set form a
+                           // thread-block cluster: partial sums are exchanged through distributed shared memory
   int32_t* slots;          // [gridDim.x][2][npad][128] raw int32 partial sums
   uint32_t* counters;      // [tiles][4], zero between launches
 };
@@ -114,8 +126,8 @@ gemm_w4a4_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
   const uint32_t pkx_bytes = (uint32_t)D.npad * PK_ROW;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < NPK; ++s) { mbar_init(pk_full(s), 1); mbar_init(pk_empty(s), 6); }
-    for (int s = 0; s < NS; ++s) { mbar_init(op_full(s), 6); mbar_init(op_empty(s), 1); }
+    for (int s = 0; s < NPK; ++s) { mbar_init(pk_full(s), 1); mbar_init(pk_empty(s), kTokWarps + 4); }
+    for (int s = 0; s < NS; ++s) { mbar_init(op_full(s), kTokWarps + 4); mbar_init(op_empty(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 4); }
     misc[1] = 0;
     fence_mbar_init();
@@ -135,7 +147,7 @@ gemm_w4a4_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
 
   // Registers: the epilogue wants the 64 accumulators of its row in registers at once, the other roles
   // need few; the warpgroups trade (see the static_assert above: the requests are covered).
-  if (warp < kConvAWarp0) reg_dec<kRegsCtl>();
+  if (warp < kConvBWarp0) reg_dec<kRegsCtl>();
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -192,23 +204,27 @@ gemm_w4a4_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
         ++seg;
       }
     }
+  } else if (warp < kConvBWarp0) {
+    // (warps 2-3: nothing to do)
   } else if (warp < kConvAWarp0) {
     // ------------------------------------------------------------------ token converters -> shared int8 tile
-    const int ctid = threadIdx.x - kConvBWarp0 * 32;     // 0..63
-    const int per_thread = D.npad / 8;                   // 16-byte chunks per thread: npad * 8 / 64
+    reg_dec<kRegsTok>();
+    constexpr int kTokThreads = kTokWarps * 32;
+    const int ctid = threadIdx.x - kConvBWarp0 * 32;     // 0..127
+    const int per_thread = D.npad * 8 / kTokThreads;     // 16-byte chunks per thread: 1, 2 or 4
     int ps = 0, s = 0; uint32_t pph = 0, ph = 0;
     for (long long g = g_begin; g < g_end; ++g) {
       if (!mbar_wait(pk_full(ps), pph, abort_flag, P.status, 7)) break;
       const uint4* src = reinterpret_cast<const uint4*>(smem + L::kPkXOff + ps * L::kPkX);
-      uint4 c[8];
+      uint4 c[4];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) if (i < per_thread) c[i] = src[i * 64 + ctid];
+      for (int i = 0; i < 4; ++i) if (i < per_thread) c[i] = src[i * kTokThreads + ctid];
       if (!mbar_wait(op_empty(s), ph ^ 1u, abort_flag, P.status, 8)) break;
       uint8_t* dst = smem + L::kB8Off + s * L::kB8Stage;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
+      for (int i = 0; i < 4; ++i) {
         if (i < per_thread) {
-          const int id = i * 64 + ctid;                  // 16-byte packed chunk: row id/8, chunk id%8
+          const int id = i * kTokThreads + ctid;         // 16-byte packed chunk: row id/8, chunk id%8
           const int r = id >> 3, ch = id & 3;            // chunks 0-3: first 128 codes, 4-7: second half
           uint32_t w[8];
           widen(c[i], w);
@@ -312,7 +328,13 @@ gemm_w4a4_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
       if (lane == 0) mbar_arrive(acc_empty(b));
 
       bool finalize = whole;
-      if (!whole) {
+      if (!whole && D.cluster > 1) {
+        // raw partial sums -> this CTA's shared memory (the packed weight ring is free: every stage has been
+        // consumed once the accumulator is complete); finished after the cluster barrier below
+        int32_t* red = reinterpret_cast<int32_t*>(smem + L::kPkWOff) + quad * 32 + lane;
+#pragma unroll
+        for (int t = 0; t < kMaxTok; ++t) if (t < npad) red[t * HR] = (int32_t)v[t];
+      } else if (!whole) {
         // raw partial sums -> this CTA's slot; the last contributor of the tile adds all slots up
         const int my_slot = (g == g_begin) ? 0 : 1;
         int32_t* slot = D.slots + ((size_t)(blockIdx.x * 2 + my_slot) * npad) * HR + quad * 32 + lane;
@@ -401,6 +423,51 @@ gemm_w4a4_decode_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_co
     }
   }
 
+  if (D.cluster > 1) {
+    // ---------------------------------------------------------------- split tiles: exchange inside the cluster
+    __syncwarp();
+    cluster_sync_all();                                  // every CTA's partial sums are in its shared memory
+    {
+      // Every thread of the CTA takes part (the other roles are done): this CTA finishes tokens
+      // [rank * tp, (rank + 1) * tp) of the tile, one (token, weight row) output per thread and pass,
+      // adding the partial sums of all CTAs of the cluster straight from their shared memory.
+      const uint32_t rank = cluster_ctarank(), csize = cluster_nctarank();
+      const int tp = D.npad / (int)csize;
+      const int t_lo = (int)rank * tp;
+      const int tile = (int)(g_begin / D.kblocks);
+      const int m_tok = P.M;
+      const size_t ldy = (size_t)P.N;
+      const uint32_t red0 = sbase + L::kPkWOff;
+      uint32_t peer[8];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) peer[c] = map_to_cta(red0, (uint32_t)c < csize ? (uint32_t)c : 0u);
+      for (int idx = threadIdx.x; idx < tp * HR; idx += kThreads) {
+        const int tok = t_lo + idx / HR, nl = idx % HR;
+        const int n = tile * HR + nl;
+        const uint32_t off = 4u * (uint32_t)(tok * HR + nl);
+        uint32_t w[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) w[c] = (uint32_t)c < csize ? ld_shared_cluster_u32(peer[c] + off) : 0u;
+        const int sum = (int)(((w[0] + w[1]) + (w[2] + w[3])) + ((w[4] + w[5]) + (w[6] + w[7])));
+        if (n < P.N && tok < m_tok) {
+          const int zw = P.wsum ? P.zero_point * __ldg(P.wsum + n) : 0;
+          const int a = (sum >> 8) - zw;
+          if (P.acc_out) P.acc_out[(size_t)tok * ldy + n] = a;
+          if (P.Y) {
+            const float ct = P.post ? __fmul_rn(P.act_scale, __ldg(P.post + tok)) : P.act_scale;
+            float y = __fmul_rn(__fmul_rn((float)a, load_scale(P.sw, P.scale_dtype, n)), ct);
+            if (P.residual) {
+              const float rs = P.res_scale ? __ldg(P.res_scale + tok) : 1.0f;
+              y = __fadd_rn(y, __fmul_rn(__bfloat162float(P.residual[(size_t)tok * ldy + n]), rs));
+            }
+            P.Y[(size_t)tok * ldy + n] = __float2bfloat16_rn(y);
+          }
+        }
+      }
+    }
+    __syncwarp();
+    cluster_sync_all();                                  // nobody leaves while a peer may still read its shared memory
+  }
   // ------------------------------------------------------------------ teardown
   __syncwarp();
   tc_fence_before();
@@ -444,6 +511,7 @@ int gemm_decode_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, co
   if (!ensure_smem_attr(attr_set, gemm_w4a4_decode_kernel, Smem::kAlloc)) return FPT_ERR_CUDA;
   DecodeParams D;
   D.g = P;
+  D.cluster = 0;
   D.npad = decode_npad(P.M);
   D.tiles = (P.N + HR - 1) / HR;
   D.kblocks = (P.K + BK - 1) / BK;
@@ -465,6 +533,11 @@ int gemm_decode_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, co
     const int max_split = D.kblocks / 2 > 0 ? D.kblocks / 2 : 1;      // at least 2 k-blocks (512 codes) per range
     if (split > max_split) split = max_split;
     ctas = D.tiles * split;
+    // a power-of-two split up to 8 that keeps at least 85 % of those CTAs: the ranges of a tile become one cluster
+    int pw = 1;
+    while (pw * 2 <= split && pw * 2 <= 8) pw *= 2;
+    D.cluster = (pw > 1 && !D.whole_tiles && pw * 100 >= split * 85 && D.kblocks % pw == 0 && D.npad % pw == 0) ? pw : 0;
+    if (D.cluster) ctas = D.tiles * pw;
     // (112 tiles stay on 112 SMs: cutting them into 148 equal ranges was measured slower, 19.4 against
     // 14.4 us at 64 tokens -- the partial sums of a split tile are 32 KB per range)
   }
@@ -472,10 +545,30 @@ int gemm_decode_launch(cudaStream_t st, const uint8_t* Xq, const uint8_t* Wq, co
   if (units < ctas) ctas = (int)units;
   D.per = (int)(D.total / ctas);
   D.rem = (int)(D.total % ctas);
-  return launch_kernel(gemm_w4a4_decode_kernel, dim3(ctas), dim3(kThreads), Smem::kAlloc, st, true, tmW, tmX, D) ==
-                 cudaSuccess
-             ? FPT_OK
-             : FPT_ERR_CUDA;
+  if (D.cluster > 1) {
+    // the clusters must fit: with one CTA per SM a cluster needs that many free SMs in one GPC
+    static PerDeviceInt fits[4];                          // cluster sizes 2, 4, 8 -> index 1, 2, 3
+    const int idx = D.cluster == 2 ? 1 : D.cluster == 4 ? 2 : 3;
+    const int cl = D.cluster;
+    const int ok = fits[idx].get([&] {
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(cl, 1, 1);
+      cfg.blockDim = dim3(kThreads, 1, 1);
+      cfg.dynamicSmemBytes = Smem::kAlloc;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = (unsigned)cl; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+      cfg.attrs = attr; cfg.numAttrs = 1;
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, gemm_w4a4_decode_kernel, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
+      return n > 0 ? n + 1 : 1;                           // 1: does not fit (cached as such)
+    }) - 1;
+    if (ok * D.cluster < ctas) D.cluster = 0;             // not all clusters resident at once: use the slots instead
+  }
+  const cudaError_t e = D.cluster > 1
+      ? launch_kernel_cluster(gemm_w4a4_decode_kernel, dim3(ctas), dim3(kThreads), Smem::kAlloc, st, true, D.cluster, tmW, tmX, D)
+      : launch_kernel(gemm_w4a4_decode_kernel, dim3(ctas), dim3(kThreads), Smem::kAlloc, st, true, tmW, tmX, D);
+  return e == cudaSuccess ? FPT_OK : FPT_ERR_CUDA;
 }
 
 }  // namespace fpt
