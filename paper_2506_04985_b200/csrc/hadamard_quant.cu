@@ -102,6 +102,131 @@ __global__ void __launch_bounds__(256) hadamard_quant_kernel(const HadQuantParam
   }
 }
 
+// The same transform for groups of 2048 channels (d_ff = 14336 = 7 x 2048) with the lane-crossing
+// stages taken off the shuffle unit: a lane first holds 64 CONSECUTIVE channels (brought in by
+// coalesced loads and redistributed through shared memory), so the stages of distance 1 ... 32 are
+// butterflies between its own registers; one transpose through shared memory (16 wide stores and
+// 32 loads per lane instead of 320 shuffles) then gives it channels
+// {64 l + 2 lane, 64 l + 2 lane + 1 : l = 0..31}, and the stages of distance 64 ... 1024 are again
+// between its own registers, two channels per packed instruction.  The order of the stages and the
+// operands of every add and subtract are those of the definition, so the codes are the same.
+// The codes return through the same shared-memory tile (a byte of two codes per lane and l) so that
+// the packed row leaves in full 128-byte lines.
+constexpr int kTrStride = 68;                        // floats per transposed row: 16-byte stores of 8 lanes hit 8 bank groups
+constexpr int kTrWarp = 32 * kTrStride;              // floats per warp
+
+template <bool kSilu>
+__global__ void __launch_bounds__(256, 3) hadamard2048_quant_kernel(const HadQuantParams P) {
+  extern __shared__ __align__(16) float tr_all[];
+  pdl_wait();                                    // the products come from the matmul before this kernel
+  pdl_launch_dependents();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int groups = P.K >> 11;
+  const long long wid = (long long)blockIdx.x * 8 + warp;
+  if (wid >= (long long)P.M * groups) return;    // (warps never meet at a CTA-wide barrier)
+  const int t = (int)(wid / groups), grp = (int)(wid % groups);
+  const uint4* row = P.X + (size_t)t * (size_t)(P.ldx >> 3);
+  float* tr = tr_all + warp * kTrWarp;
+  // The group's 256 chunks of 8 channels arrive in fully coalesced loads (lane l takes chunks
+  // 32 j + l) and are parked in the tile; then every lane picks up ITS 64 consecutive channels
+  // (chunks 8 l ... 8 l + 7).  Chunk c sits at row c / 8, position (c % 8) ^ (row % 8): both the
+  // stores and the loads of a quarter warp then cover all eight 16-byte bank groups.
+  uint4* stage = reinterpret_cast<uint4*>(tr);
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int c = 32 * j + lane;                 // chunk of the group
+    uint4 v;
+    if (kSilu) {
+      // products chunk grp * 256 + c: its gate chunk, the up chunk 8 further
+      const int pc = grp * 256 + c;
+      const uint4* g = row + ((pc >> 3) << 4) + (pc & 7);
+      const uint4 gv = __ldg(g), uv = __ldg(g + 8);
+      v.x = silu_mul_pair(gv.x, uv.x); v.y = silu_mul_pair(gv.y, uv.y);
+      v.z = silu_mul_pair(gv.z, uv.z); v.w = silu_mul_pair(gv.w, uv.w);
+    } else {
+      v = __ldg(row + grp * 256 + c);
+    }
+    const int r = c >> 3;
+    stage[r * 8 + ((c & 7) ^ (r & 7))] = v;
+  }
+  __syncwarp();
+  float x[64];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const uint4 v = stage[lane * 8 + (j ^ (lane & 7))];
+    x[8 * j + 0] = bf16lo_to_f32(v.x); x[8 * j + 1] = bf16hi_to_f32(v.x);
+    x[8 * j + 2] = bf16lo_to_f32(v.y); x[8 * j + 3] = bf16hi_to_f32(v.y);
+    x[8 * j + 4] = bf16lo_to_f32(v.z); x[8 * j + 5] = bf16hi_to_f32(v.z);
+    x[8 * j + 6] = bf16lo_to_f32(v.w); x[8 * j + 7] = bf16hi_to_f32(v.w);
+  }
+  __syncwarp();                                  // the tile is reused for the transpose below
+  // distance 1
+#pragma unroll
+  for (int i = 0; i < 64; i += 2) {
+    const float a = x[i], b = x[i + 1];
+    x[i] = __fadd_rn(a, b);
+    x[i + 1] = __fsub_rn(a, b);
+  }
+  // distances 2 ... 32, two butterflies per instruction
+#pragma unroll
+  for (int s = 2; s < 64; s <<= 1)
+#pragma unroll
+    for (int i = 0; i < 64; i += 2)
+      if ((i & s) == 0) {
+        const uint64_t a = pack_f32x2(x[i], x[i + 1]), b = pack_f32x2(x[i + s], x[i + s + 1]);
+        unpack_f32x2(add_f32x2(a, b), x[i], x[i + 1]);
+        unpack_f32x2(sub_f32x2(a, b), x[i + s], x[i + s + 1]);
+      }
+  // transpose: row `lane` of the tile <- this lane's 64 values; then column pair `lane` of every row
+#pragma unroll
+  for (int j = 0; j < 16; ++j)
+    *reinterpret_cast<float4*>(tr + lane * kTrStride + 4 * j) = make_float4(x[4 * j], x[4 * j + 1], x[4 * j + 2], x[4 * j + 3]);
+  __syncwarp();
+#pragma unroll
+  for (int l = 0; l < 32; ++l) {
+    const float2 v = *reinterpret_cast<const float2*>(tr + l * kTrStride + 2 * lane);
+    x[2 * l] = v.x; x[2 * l + 1] = v.y;          // channels 64 l + 2 lane, 64 l + 2 lane + 1
+  }
+  // distances 64 ... 1024: between rows l and l + d
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1)
+#pragma unroll
+    for (int l = 0; l < 32; ++l)
+      if ((l & d) == 0) {
+        const uint64_t a = pack_f32x2(x[2 * l], x[2 * l + 1]), b = pack_f32x2(x[2 * (l + d)], x[2 * (l + d) + 1]);
+        unpack_f32x2(add_f32x2(a, b), x[2 * l], x[2 * l + 1]);
+        unpack_f32x2(sub_f32x2(a, b), x[2 * (l + d)], x[2 * (l + d) + 1]);
+      }
+  const float p = P.s_in ? __ldg(P.s_in + t) : 1.0f;
+  const QuantConsts qc = quant_consts(p, P.inv_delta, P.qmax_minus_z, P.flip);
+  __syncwarp();                                  // every lane has read the tile before it is overwritten
+  uint8_t* bytes = reinterpret_cast<uint8_t*>(tr);
+#pragma unroll
+  for (int l = 0; l < 32; ++l) {
+    const float h0 = __fmul_rn(x[2 * l], P.norm), h1 = __fmul_rn(x[2 * l + 1], P.norm);
+    bytes[l * 36 + lane] = (uint8_t)((quant_pair_f32(h0, h1, qc, 0u) ^ qc.flip) & 0xFFu);     // two codes
+  }
+  __syncwarp();
+  uint32_t* out = P.Xq + (size_t)t * (size_t)(P.K >> 3) + grp * 256;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int w = i * 32 + lane;                 // word w: codes of channels 8 w ... 8 w + 7 = row w / 8, bytes 4 (w % 8) ...
+    out[w] = *reinterpret_cast<const uint32_t*>(bytes + (w >> 3) * 36 + 4 * (w & 7));
+  }
+}
+
+static cudaError_t launch_had2048(const HadQuantParams& P, cudaStream_t st) {
+  const long long warps = (long long)P.M * (P.K / 2048);
+  const size_t smem = (size_t)8 * kTrWarp * sizeof(float);
+  static PerDeviceInt attr_a, attr_b;
+  if (P.silu_inter) {
+    if (!ensure_smem_attr(attr_a, hadamard2048_quant_kernel<true>, (int)smem)) return cudaErrorInvalidValue;
+    return launch_kernel(hadamard2048_quant_kernel<true>, dim3((unsigned)((warps + 7) / 8)), dim3(256), smem, st, true, P);
+  }
+  if (!ensure_smem_attr(attr_b, hadamard2048_quant_kernel<false>, (int)smem)) return cudaErrorInvalidValue;
+  return launch_kernel(hadamard2048_quant_kernel<false>, dim3((unsigned)((warps + 7) / 8)), dim3(256), smem, st, true, P);
+}
+
 template <int C>
 static cudaError_t launch_had(const HadQuantParams& P, cudaStream_t st) {
   const long long warps = (long long)P.M * (P.K / (256 * C));
@@ -129,7 +254,7 @@ cudaError_t hadamard_quant_launch(cudaStream_t st, const void* X, int M, int K, 
     case 256: return launch_had<1>(P, st);
     case 512: return launch_had<2>(P, st);
     case 1024: return launch_had<4>(P, st);
-    case 2048: return launch_had<8>(P, st);
+    case 2048: return launch_had2048(P, st);
     case 4096: return launch_had<16>(P, st);
     default: return cudaErrorInvalidValue;
   }

@@ -50,7 +50,19 @@ __device__ __forceinline__ uint64_t mul_f32x2(uint64_t a, uint64_t b) {
   asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
   return r;
 }
-// (There is no packed add here on purpose.  The quantiser needs the product (x * p) * (1/D) ROUNDED
+// Packed add / subtract: used only where no multiply feeds them (the butterflies of the Hadamard
+// kernel), so there is nothing a compiler could contract them with.
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t sub_f32x2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+// (There is no packed add in the quantiser on purpose.  The quantiser needs the product (x * p) * (1/D) ROUNDED
 // before the rounding constant is added; a packed multiply followed by a packed add was contracted
 // into one fused multiply-add -- the explicit .rn of the packed forms does not stop that -- and a
 // product that rounds to exactly k + 1/2 from slightly off it then took the other code.  The scalar
