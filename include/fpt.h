@@ -363,6 +363,18 @@ int fpt_decoder_attn_out(void* stream, const void* A, int M, int k_o,
 int fpt_probe_mma(void* stream, int pair, int n, int n_acc, int a_in_tmem, int iters, int ctas,
                   unsigned long long* cycles, void* workspace);
 
+/*
+ * Self-test of the bounded device-side wait (the paper has no counterpart).  Every wait inside the
+ * kernels gives up after a time limit, records a code in the status word of the workspace and lets
+ * the kernel end normally (FPT_ERR_TIMEOUT from fpt_check_status).  This call runs that very wait
+ * routine in a one-warp kernel on a barrier nothing ever arrives at, with a limit of limit_us
+ * microseconds (1 .. 100000): the kernel ends by itself after that time.
+ *   workspace  device, 16-byte aligned, at least 8192 bytes, status word zero (fpt_reset_status)
+ *   gave_up    device, may be NULL: 1 if the wait returned "gave up"
+ * Afterwards fpt_check_status(stream, workspace) returns FPT_ERR_TIMEOUT until fpt_reset_status.
+ */
+int fpt_selftest_wait_timeout(void* stream, void* workspace, unsigned int limit_us, unsigned int* gave_up);
+
 /* Bytes of caller-provided scratch an entry point needs (op = FPT_OP_*).
  * FPT_OP_LINEAR / FPT_OP_GEMM / FPT_OP_GEMM_A8 / FPT_OP_LINEAR_A8: (M, N, K); FPT_OP_MLP: (M, d_ff, d). */
 size_t fpt_workspace_bytes(int op, int M, int N, int K);

@@ -25,7 +25,7 @@ EXPORTS = ["fpt_version", "fpt_strerror", "fpt_quantize_weights", "fpt_interleav
            "fpt_w4a4_gemm", "fpt_w4a4_linear", "fpt_w4a4_linear_static", "fpt_decoder_mlp", "fpt_decoder_attn_qkv",
            "fpt_decoder_attn_out", "fpt_act_quant_dynamic", "fpt_w4a4_linear_dynamic", "fpt_w4a8_gemm", "fpt_workspace_bytes",
            "fpt_reset_status",
-           "fpt_check_status", "fpt_probe_mma", "fpt_set_programmatic_launch"]
+           "fpt_check_status", "fpt_probe_mma", "fpt_set_programmatic_launch", "fpt_selftest_wait_timeout"]
 
 
 class QParams(ctypes.Structure):
@@ -90,6 +90,7 @@ def lib():
         L.fpt_reset_status.argtypes = [vp, vp]
         L.fpt_check_status.argtypes = [vp, vp]
         L.fpt_set_programmatic_launch.argtypes = [ci]
+        L.fpt_selftest_wait_timeout.argtypes = [vp, vp, ctypes.c_uint, vp]
         L.fpt_probe_mma.argtypes = [vp, ci, ci, ci, ci, ci, ci, vp, vp]
         for name in EXPORTS:
             if name not in ("fpt_strerror", "fpt_workspace_bytes", "fpt_version"):
@@ -348,3 +349,10 @@ def fpt_probe_mma(pair, n, n_acc, a_in_tmem, iters, ctas, ws=None, want_cycles=T
 def fpt_set_programmatic_launch(enabled):
     """Switches programmatic dependent launch of the library's kernels on or off; returns the previous setting."""
     return lib().fpt_set_programmatic_launch(int(bool(enabled)))
+
+
+def fpt_selftest_wait_timeout(ws, limit_us=1000):
+    """Runs the library's bounded wait on a barrier nothing arrives at -> uint32 tensor [1]: 1 if it gave up."""
+    flag = torch.zeros((1,), dtype=torch.int32, device=ws.device)
+    _check(lib().fpt_selftest_wait_timeout(_stream(), _ptr(ws), int(limit_us), _ptr(flag)), "fpt_selftest_wait_timeout")
+    return flag

@@ -113,10 +113,38 @@ __global__ void __launch_bounds__(kThreads, 1) mma_probe_kernel(const Params P) 
   }
 }
 
+// Self-test of the bounded wait every kernel of the library relies on: one thread waits on an
+// mbarrier on which nothing ever arrives, with a limit of `limit_ns`; the wait must give up, record
+// where in the status word, and the kernel must end normally.
+__global__ void __launch_bounds__(32, 1) wait_timeout_kernel(uint32_t* status, unsigned long long limit_ns, uint32_t* gave_up) {
+  __shared__ __align__(8) unsigned long long bar_mem;
+  __shared__ uint32_t abort_flag;
+  const uint32_t bar = smem_u32(&bar_mem);
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(bar, 1);
+    fence_mbar_init();
+  }
+  __syncwarp();
+  if (threadIdx.x == 0) {
+    const bool ok = mbar_wait_limit(bar, 0, &abort_flag, status, 14, limit_ns);
+    if (gave_up) *gave_up = ok ? 0u : 1u;
+    mbar_inval(bar);
+  }
+}
+
 }  // namespace probe
 }  // namespace fpt
 
 using namespace fpt;
+
+extern "C" int fpt_selftest_wait_timeout(void* stream, void* workspace, unsigned int limit_us, unsigned int* gave_up) {
+  if (!workspace || limit_us == 0 || limit_us > 100000u) return FPT_ERR_BAD_ARG;
+  if ((uintptr_t)workspace & 15) return FPT_ERR_ALIGNMENT;
+  probe::wait_timeout_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(reinterpret_cast<uint32_t*>(workspace),
+                                                                (unsigned long long)limit_us * 1000ull, gave_up);
+  return cudaGetLastError() == cudaSuccess ? FPT_OK : FPT_ERR_CUDA;
+}
 
 extern "C" int fpt_probe_mma(void* stream, int pair, int n, int n_acc, int a_in_tmem, int iters, int ctas,
                              unsigned long long* cycles, void* workspace) {

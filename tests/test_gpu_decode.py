@@ -86,3 +86,17 @@ def test_decode_extreme_codes_and_long_k():
 def test_decode_many_tiles_without_counters():
     """More 128-row tiles than the control block has counters: ranges then end on tile boundaries."""
     _run(8, 64000, 128, seed=11)
+
+
+@pytest.mark.parametrize("M,N,K,what", [
+    (40, 8192, 2048, "64 tiles cut in 2: clusters of two CTAs"),
+    (33, 2048, 4096, "16 tiles cut in 8: clusters of eight CTAs"),
+    (64, 4096, 2048, "32 tiles cut in 4, asymmetric grid and residual below"),
+    (64, 1024, 8192, "8 tiles cut in 16 ranges: no cluster that size, partial sums through the scratch slots"),
+    (20, 1152, 1280, "9 tiles, 5 k-blocks: ranges that do not end on tile boundaries")])
+def test_decode_split_tiles_cluster_and_slot_paths(M, N, K, what):
+    """Few tiles and long rows: every tile is cut into ranges whose partial sums are exchanged through a
+    cluster's shared memory (2, 4, 8 CTAs) or through scratch slots; twice on one workspace."""
+    ws = B.new_workspace(B.OP_GEMM, M, N, K)
+    _run(M, N, K, seed=21, ws=ws, reps=2)
+    _run(M, N, K, symmetric=False, z=9, seed=22, post=True, residual=True, f16=False, ws=ws, reps=2)
