@@ -16,9 +16,9 @@
 // Roles per CTA (20 warps):
 //   warp 0        TMA producer: packed tiles (128 rows x 64 bytes of each operand per k-block)
 //   warp 1        tensor-memory owner; in the leader CTA (rank 0) also the MMA issuer
-//   warps 4..7    activation converters: shared -> registers -> widen -> tcgen05.st (one row per thread);
-//                 while that store completes they also widen the last quarter of the weight tile
-//   warps 8..11   weight converters: shared -> widen -> 128-byte-swizzled K-major int8 tile (three quarters)
+//   warps 4..11   converters, two groups of four warps that take the k-blocks in turns: a group widens
+//                 the CTA's activation rows (shared -> registers -> tcgen05.st, one row per thread) and,
+//                 while that store completes, its weight rows (-> 128-byte-swizzled K-major int8 tile)
 //   warps 12..19  epilogue: tcgen05.ld, >> 8, scales, bf16 into a swizzled shared-memory tile; the
 //                 accumulator is released as soon as it has been read, the tile leaves by TMA store;
 //                 a residual tile is fetched by TMA into the same slabs while the tile's matmul runs
@@ -42,13 +42,13 @@ constexpr int kAccCols = 256;              // tensor-memory columns of the accum
 constexpr int kAStageCols = BK / 4;        // 32 columns hold 128 int8 per lane
 constexpr int kTmemCols = 512;
 constexpr int kThreads = 640;
-constexpr int kConvAWarp0 = 4, kConvBWarp0 = 8, kEpiWarp0 = 12, kEpiWarps = 8;
+constexpr int kConvWarp0 = 4, kEpiWarp0 = 12, kEpiWarps = 8;
 // Registers per thread: what the CTA is launched with, and what the roles trade it into (warps 0-3,
-// activation converters, weight converters, epilogue).  A CTA can only redistribute what it owns: an
+// the two converter groups, epilogue).  A CTA can only redistribute what it owns: an
 // increase that the decreases do not cover would never return, so the sum is checked here.
-constexpr int kRegsLaunch = 96, kRegsCtl = 48, kRegsConvA = 56, kRegsConvB = 56, kRegsEpi = 152;
+constexpr int kRegsLaunch = 96, kRegsCtl = 48, kRegsConv = 64, kRegsEpi = 152;
 static_assert(kThreads * kRegsLaunch <= 65536, "launch allocation exceeds the register file");
-static_assert(128 * (kRegsCtl + kRegsConvA + kRegsConvB) + 32 * kEpiWarps * kRegsEpi <= kThreads * kRegsLaunch,
+static_assert(128 * (kRegsCtl + 2 * kRegsConv) + 32 * kEpiWarps * kRegsEpi <= kThreads * kRegsLaunch,
               "the warpgroups ask for more registers than the CTA was launched with: setmaxnreg.inc would never return");
 
 // NS: stages of widened operands (int8 weight tile in shared memory + activation columns in
@@ -114,8 +114,6 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
   __nv_bfloat16* const y_out_p = P.Y;
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  // quarters of the weight tile the weight converters widen; the activation converters take the rest
-  constexpr int kBShare = kA8 ? 4 : 3;
   const uint32_t rank = cluster_ctarank();             // 0 = leader
   const int pair_id = blockIdx.x >> 1;
   const int num_pairs = gridDim.x >> 1;
@@ -127,8 +125,8 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
   constexpr int hb = tn >> 1;                          // weight rows of the tile this CTA holds
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < NPK; ++s) { mbar_init(pk_full(s), 1); mbar_init(pk_empty(s), 8); }
-    for (int s = 0; s < NS; ++s) { mbar_init(op_full(s), 16); mbar_init(op_empty(s), 1); }
+    for (int s = 0; s < NPK; ++s) { mbar_init(pk_full(s), 1); mbar_init(pk_empty(s), 4); }      // the four warps of a group
+    for (int s = 0; s < NS; ++s) { mbar_init(op_full(s), 8); mbar_init(op_empty(s), 1); }        // ... in both CTAs
     mbar_init(acc_full, 1);
     mbar_init(acc_empty, 2 * kEpiWarps);
     for (int b = 0; b < 2; ++b) { mbar_init(sc_full(b), kEpiWarps); mbar_init(stg_full(b), 4); mbar_init(stg_empty(b), 1); mbar_init(res_full(b), 1); }
@@ -153,10 +151,10 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
 
   // Registers: the epilogue wants the 128 accumulators of its row in registers at once, the other
   // roles need few; the warpgroups trade.  A CTA can only redistribute what it was launched with
-  // (640 x 96 registers): 128 x (48 + 56 + 56) + 256 x 152 = 59392 <= 61440, so the request of the
+  // (640 x 96 registers): 128 x (48 + 64 + 64) + 256 x 152 = 61440 <= 61440, so the request of the
   // epilogue groups is always met once the three other groups have given theirs back.  Each role
   // branch starts with its own re-allocation (the compiler budgets registers per branch).
-  if (warp < kConvAWarp0) {
+  if (warp < kConvWarp0) {
     reg_dec<kRegsCtl>();
     if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -210,108 +208,83 @@ gemm_w4a4_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
       }
     }
     }
-  } else if (warp < kConvBWarp0) {
-    // ------------------------------------------------------------------ activation converters -> tensor memory
-    reg_dec<kRegsConvA>();
-    const int quad = warp - kConvAWarp0;                 // == warp % 4: the TMEM lanes this warp may touch
-    const int r = quad * 32 + lane;                      // row of the CTA's 128
+  } else if (warp < kEpiWarp0) {
+    // ------------------------------------------------------------------ converters
+    // Two groups of four warps (4..7 and 8..11) take the k-blocks in turns, and a group widens a whole
+    // k-block: the CTA's 128 activation rows into tensor memory (one row per thread; warp % 4 selects
+    // the tensor-memory lanes the warp may touch) and the CTA's weight rows into the int8 tile in shared
+    // memory.  For one warp a k-block is a chain of long latencies (shared loads, the tensor-memory store
+    // and its wait, the proxy fence) that does not shrink with the tile; alternating groups give every
+    // chain two k-block periods.
+    reg_dec<kRegsConv>();
+    const int grp = (warp - kConvWarp0) >> 2;
+    const int quad = warp & 3;                           // the TMEM lanes this warp may touch
+    const int r = quad * 32 + lane;                      // activation row of the CTA's 128; also this thread's chunk column
     const uint32_t swz = (uint32_t)((r >> 1) & 3);       // SWIZZLE_64B: 16-byte chunk index ^= (row / 2) % 4
     const uint32_t op_full_leader = map_to_cta(op_full(0), 0);
     int ps = 0, s = 0; uint32_t pph = 0, ph = 0;
+    uint32_t gk = 0;                                     // k-blocks since the start of the kernel
     bool ok = true;
     for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs) {
-      for (int kb = 0; kb < kblocks; ++kb) {
-        if (!mbar_wait(pk_full(ps), pph, abort_flag, status_w, 5)) { ok = false; break; }
-        uint32_t v[32];
-        uint4 cb = make_uint4(0, 0, 0, 0);
-        if constexpr (kA8) {
-          // int8 codes, 128-byte rows under the 128-byte swizzle.  The weight side orders the 32 codes
-          // of a group as 16 even-k then 16 odd-k bytes (that is how the nibbles fall apart); the
-          // activation bytes are put into the same order.
-          const uint8_t* src = smem + L::kPkAOff + ps * L::kPkOpA + r * I8_ROW;
+      for (int kb = 0; kb < kblocks; ++kb, ++gk) {
+        if ((int)(gk & 1u) == grp) {
+          if (!mbar_wait(pk_full(ps), pph, abort_flag, status_w, 5)) { ok = false; break; }
+          uint32_t v[32];
+          if constexpr (kA8) {
+            // int8 codes, 128-byte rows under the 128-byte swizzle.  The weight side orders the 32 codes
+            // of a group as 16 even-k then 16 odd-k bytes (that is how the nibbles fall apart); the
+            // activation bytes are put into the same order.
+            const uint8_t* src = smem + L::kPkAOff + ps * L::kPkOpA + r * I8_ROW;
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            const uint4 c0 = *reinterpret_cast<const uint4*>(src + (((uint32_t)(2 * g) ^ (uint32_t)(r & 7)) << 4));
-            const uint4 c1 = *reinterpret_cast<const uint4*>(src + (((uint32_t)(2 * g + 1) ^ (uint32_t)(r & 7)) << 4));
-            const uint32_t a[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+            for (int g = 0; g < 4; ++g) {
+              const uint4 c0 = *reinterpret_cast<const uint4*>(src + (((uint32_t)(2 * g) ^ (uint32_t)(r & 7)) << 4));
+              const uint4 c1 = *reinterpret_cast<const uint4*>(src + (((uint32_t)(2 * g + 1) ^ (uint32_t)(r & 7)) << 4));
+              const uint32_t a[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
 #pragma unroll
-            for (int w = 0; w < 4; ++w) {
-              v[8 * g + w] = __byte_perm(a[2 * w], a[2 * w + 1], 0x6420);
-              v[8 * g + 4 + w] = __byte_perm(a[2 * w], a[2 * w + 1], 0x7531);
+              for (int w = 0; w < 4; ++w) {
+                v[8 * g + w] = __byte_perm(a[2 * w], a[2 * w + 1], 0x6420);
+                v[8 * g + 4 + w] = __byte_perm(a[2 * w], a[2 * w + 1], 0x7531);
+              }
             }
+          } else {
+            const uint8_t* src = smem + L::kPkAOff + ps * L::kPkOpA + r * PK_ROW;
+            uint4 c[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) c[j] = *reinterpret_cast<const uint4*>(src + (((uint32_t)j ^ swz) << 4));
+#pragma unroll
+            for (int j = 0; j < 4; ++j) widen(c[j], v + 8 * j);
           }
-        } else {
-          const uint8_t* src = smem + L::kPkAOff + ps * L::kPkOpA + r * PK_ROW;
-          uint4 c[4];
+          // the packed weight tile: 16-byte chunk i * 128 + r is row (i * 128 + r) / 4, chunk r % 4
+          const uint4* srcb = reinterpret_cast<const uint4*>(smem + L::kPkBOff + ps * L::kPkOp);
+          uint4 cb[4];
 #pragma unroll
-          for (int j = 0; j < 4; ++j) c[j] = *reinterpret_cast<const uint4*>(src + (((uint32_t)j ^ swz) << 4));
-          cb = reinterpret_cast<const uint4*>(smem + L::kPkBOff + ps * L::kPkOp)[kBShare * 128 + r];
+          for (int i = 0; i < 4; ++i) cb[i] = srcb[i * 128 + r];
+          if (!mbar_wait(op_empty(s), ph ^ 1u, abort_flag, status_w, 6)) { ok = false; break; }
+          tc_fence_after();
+          tmem_st_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + kAccCols + s * kAStageCols, v);
+          // while the tensor-memory store completes: the weight rows
+          uint8_t* dst = smem + L::kB8Off + s * L::kB8Stage;
 #pragma unroll
-          for (int j = 0; j < 4; ++j) widen(c[j], v + 8 * j);
-        }
-        if (!mbar_wait(op_empty(s), ph ^ 1u, abort_flag, status_w, 6)) { ok = false; break; }
-        tc_fence_after();
-        tmem_st_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + kAccCols + s * kAStageCols, v);
-        if constexpr (!kA8) {
-          // While the tensor-memory store completes: this warp's share of the WEIGHT tile (its last 32
-          // rows).  The weight converters are the busiest role (measured: 74 % of the k-block period
-          // against 48 % here), so a quarter of their tile is widened by these warps instead.
-          const int id = kBShare * 128 + r;              // 16-byte packed chunk: row id/4, chunk id%4
-          const int br = id >> 2, ch = id & 3;
-          if (br < hb) {                                 // a narrower tile has fewer weight rows
+          for (int i = 0; i < 4; ++i) {
+            const int br = (i * 128 + r) >> 2, ch = r & 3;
+            if (i == 3 && br >= hb) continue;            // a narrower tile has fewer weight rows
             uint32_t w[8];
-            widen(cb, w);
-            uint8_t* rowp = smem + L::kB8Off + s * L::kB8Stage + br * I8_ROW;
+            widen(cb[i], w);
+            uint8_t* rowp = dst + br * I8_ROW;
             *reinterpret_cast<uint4*>(rowp + (((2 * ch) ^ (br & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
             *reinterpret_cast<uint4*>(rowp + (((2 * ch + 1) ^ (br & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
           }
+          tmem_wait_st();
+          tc_fence_before();
+          // One fence for both hand-overs: the widened tile becomes visible to the tensor core's async
+          // proxy, and the reads of the packed tiles (consumed by the stores above) are ordered before
+          // the TMA writes that re-fill them.  The packed tiles go back to TMA only here: handing them
+          // back right after the loads, with nothing depending on them yet, let the next TMA write
+          // overtake reads still in flight (seen as wrong weight rows, rarely, under load).
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) { mbar_arrive(pk_empty(ps)); mbar_arrive_cluster(op_full_leader + 8u * s); }
         }
-        tmem_wait_st();
-        tc_fence_before();
-        // The packed tile goes back to TMA only here: its reads have been consumed (the store above
-        // depends on them) and are fenced against the async proxy, which will overwrite the tile.
-        // Handing it back right after the loads, with nothing depending on them yet, let the next
-        // TMA write overtake reads still in flight (seen as wrong weight rows, rarely, under load).
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) { mbar_arrive(pk_empty(ps)); mbar_arrive_cluster(op_full_leader + 8u * s); }
-        if (++ps == NPK) { ps = 0; pph ^= 1u; }
-        if (++s == NS) { s = 0; ph ^= 1u; }
-      }
-    }
-  } else if (warp < kEpiWarp0) {
-    // ------------------------------------------------------------------ weight converters -> shared int8 tile
-    reg_dec<kRegsConvB>();
-    const int ctid = threadIdx.x - kConvBWarp0 * 32;     // 0..127
-    const uint32_t op_full_leader = map_to_cta(op_full(0), 0);
-    int ps = 0, s = 0; uint32_t pph = 0, ph = 0;
-    bool ok = true;
-    for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs) {
-      for (int kb = 0; kb < kblocks; ++kb) {
-        if (!mbar_wait(pk_full(ps), pph, abort_flag, status_w, 7)) { ok = false; break; }
-        const uint4* src = reinterpret_cast<const uint4*>(smem + L::kPkBOff + ps * L::kPkOp);
-        uint4 c[kBShare];
-#pragma unroll
-        for (int i = 0; i < kBShare; ++i) c[i] = src[i * 128 + ctid];
-        if (!mbar_wait(op_empty(s), ph ^ 1u, abort_flag, status_w, 8)) { ok = false; break; }
-        uint8_t* dst = smem + L::kB8Off + s * L::kB8Stage;
-#pragma unroll
-        for (int i = 0; i < kBShare; ++i) {
-          const int id = i * 128 + ctid;                 // 16-byte packed chunk: row id/4, chunk id%4
-          const int r = id >> 2, ch = id & 3;
-          if (i == 3 && r >= hb) continue;               // (int8 activations: this role has all four quarters)
-          uint32_t w[8];
-          widen(c[i], w);
-          uint8_t* rowp = dst + r * I8_ROW;
-          *reinterpret_cast<uint4*>(rowp + (((2 * ch) ^ (r & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-          *reinterpret_cast<uint4*>(rowp + (((2 * ch + 1) ^ (r & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
-        }
-        // one fence for both hand-overs: the widened tile becomes visible to the tensor core's async
-        // proxy, and the reads of the packed tile (consumed by the stores above) are ordered before
-        // the TMA write that re-fills it
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) { mbar_arrive(pk_empty(ps)); mbar_arrive_cluster(op_full_leader + 8u * s); }
         if (++ps == NPK) { ps = 0; pph ^= 1u; }
         if (++s == NS) { s = 0; ph ^= 1u; }
       }
