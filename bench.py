@@ -33,7 +33,7 @@ EPS = 1e-5
 NSETS = 4
 # dram__bytes_read.sum + dram__bytes_write.sum of one fused-QKV matmul launch, from the ncu capture
 # summarised in profiles/gemm_w4a4_pair_2048x6144x4096.md (set to None when the kernel changes)
-GEMM_QKV_DRAM_BYTES = 16.98e6
+GEMM_QKV_DRAM_BYTES = 17.04e6
 METRIC = "W4A4 linear TOPS (prefill, Llama-3-8B-shaped attention projections, 2048 tokens)"
 
 
@@ -293,20 +293,27 @@ def run_gpu(args):
         torch.cuda.synchronize()
 
     def capture(fn):
-        """One CUDA graph per operand set: the launches of `fn(S)` without the host's per-call cost."""
+        """The launches of `fn(S)` without the host's per-call cost: one CUDA graph that runs fn on every
+        operand set in turn (as a model's forward pass holds many layers in one graph, so that a kernel's
+        set-up overlaps the tail of the kernel before it across the whole chain), plus one single-set graph
+        per set for a remainder."""
         graphs = []
-        for S in sets:
+        for group in [sets] + [[S] for S in sets]:
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g):
-                fn(S)
+                for S in group:
+                    fn(S)
             graphs.append(g)
         return graphs
 
     def timed(graphs, n):
+        """Exactly n executions of fn, each on the next operand set of the rotation."""
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        for i in range(n):
-            graphs[i % NSETS].replay()
+        for _ in range(n // NSETS):
+            graphs[0].replay()
+        for i in range(n % NSETS):
+            graphs[1 + i].replay()
         e1.record()
         torch.cuda.synchronize()
         return e0.elapsed_time(e1)
@@ -316,8 +323,8 @@ def run_gpu(args):
         step(sets[i % NSETS])                        # eager: also sets the kernels' attributes before capture
     torch.cuda.synchronize()
     step_graphs = capture(step)
-    for i in range(NSETS):
-        step_graphs[i].replay()
+    for g in step_graphs:
+        g.replay()
     barrier()
     sampler = ClockSampler(local)
     sampler.start()
@@ -393,7 +400,8 @@ def run_gpu(args):
     h2d = 2 * M_TOK * HID * 2
     d2h = M_TOK * (N_QKV + N_O) * 2
 
-    # ---- per-kernel pass: each of the step's four kernels alone, replayed over the rotating sets;
+    # ---- per-kernel pass: each of the step's four kernels alone, replayed over the rotating sets (a graph
+    # holds one launch per set, so a launch follows a launch of the same kernel on other operands);
     # its length does not depend on --steps: 240 replays per run, median of 5 runs ----
     from paper_2506_04985_b200 import microbench as MB
     KREPLAYS, KRUNS = 240, 5
@@ -522,7 +530,7 @@ def run_gpu(args):
                 "e2e": {"value": e2e_tops, "unit": "TOPS", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                         "steps": e2e_steps, "mode": "eager calls through the binding; upload, compute and download "
                                                     "of consecutive steps overlap on three streams"},
-                "gpu_launches": 4 * args.steps, "launch_mode": "one CUDA graph per step (4 kernels), replayed",
+                "gpu_launches": 4 * args.steps, "launch_mode": f"CUDA graphs of {NSETS} steps (one per operand set, 4 kernels each), replayed",
                 "clocks": clocks, "roofline": roofline, "kernel_us": kern_us, "other_configs": other,
                 "cpu_baseline": {"value": cpu_tops, "unit": "TOPS", "cores": blas_threads(), "kind": "oracle",
                                  "sample": f"{rows} of {M_TOK} token rows x all {N_QKV + N_O} output columns, "
