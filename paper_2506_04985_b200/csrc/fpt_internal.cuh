@@ -30,9 +30,6 @@ struct GemmParams {
   float mid_inv_delta;         // 1/D of the grid at the down-projection input
   int mid_qmax_minus_z;
   uint32_t mid_flip;
-  int early_weights;           // Wq / sw / wsum are certainly not written by the kernel in front of this one in
-                               // the stream (the library's own quantiser): a kernel may request them before
-                               // its dependency wait
   uint32_t* status;            // control block of the workspace (status word, decode counters)
   void* scratch;               // gemm_scratch_bytes(M) bytes behind the control block (decode partial sums)
 };
