@@ -117,6 +117,18 @@ __device__ __forceinline__ uint32_t quant_pair_f32(float x0, float x1, const Qua
   return (prev * 16u + c1) * 16u + c0;
 }
 
+// The same for a packed pair that is first multiplied by `pre2` (each lane rounded on its own): three
+// packed multiplies, nothing a compiler could contract.
+__device__ __forceinline__ uint32_t quant_pair_f32_pre(uint64_t x2, uint64_t pre2, const QuantConsts& c, uint32_t prev) {
+  float v0, v1;
+  unpack_f32x2(mul_f32x2(mul_f32x2(mul_f32x2(x2, pre2), c.np2), c.d2), v0, v1);
+  v0 = __fadd_rn(v0, 12582912.0f);
+  v1 = __fadd_rn(v1, 12582912.0f);
+  const uint32_t c0 = (uint32_t)__viaddmin_s32_relu(max(__float_as_int(v0), 0), c.bias, 15);
+  const uint32_t c1 = (uint32_t)__viaddmin_s32_relu(max(__float_as_int(v1), 0), c.bias, 15);
+  return (prev * 16u + c1) * 16u + c0;
+}
+
 // Eight float32 values -> eight packed codes (value 0 in bits 0-3).
 __device__ __forceinline__ uint32_t quant_word_f32(const float (&x)[8], const QuantConsts& c) {
   uint32_t w = quant_pair_f32(x[6], x[7], c, 0u);
