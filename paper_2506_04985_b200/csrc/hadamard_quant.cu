@@ -201,8 +201,8 @@ __global__ void __launch_bounds__(256, 3) hadamard2048_quant_kernel(const HadQua
   const QuantConsts qc = quant_consts(p, P.inv_delta, P.qmax_minus_z, P.flip);
   __syncwarp();                                  // every lane has read the tile before it is overwritten
   uint8_t* bytes = reinterpret_cast<uint8_t*>(tr);
-#pragma unroll
   const uint64_t norm2 = pack_f32x2(P.norm, P.norm);
+#pragma unroll
   for (int l = 0; l < 32; ++l)                   // h = x * norm, then the quantiser: two codes per byte
     bytes[l * 36 + lane] = (uint8_t)((quant_pair_f32_pre(pack_f32x2(x[2 * l], x[2 * l + 1]), norm2, qc, 0u) ^ qc.flip) & 0xFFu);
   __syncwarp();
