@@ -463,7 +463,7 @@ def run_gpu(args):
         def measure(kind, M, N, K, reps, f16=False):
             nsets = max(2, min(8, int(300e6 / max(1.0, N * K / 2 + M * K / 2 + 2.0 * M * N))))
             runs, ops, nbytes = MB.make_case(kind, M, N, K, nsets, dev, f16)
-            us = MB.time_case_graph(runs, reps)
+            us = float(np.median([MB.time_case_graph(runs, reps) for _ in range(3)]))
             del runs
             torch.cuda.empty_cache()
             return us, ops, nbytes
@@ -501,7 +501,7 @@ def run_gpu(args):
         for name, kind, bits in (("static W4A4", "linear", 4), ("dynamic W4A4", "linear_dynamic", 4),
                                  ("dynamic W4A8", "linear_dynamic", 8)):
             runs, ops, _ = MB.make_case(kind, M_TOK, N_QKV, HID, 4, dev, False, bits)
-            us = MB.time_case_graph(runs, 20)
+            us = float(np.median([MB.time_case_graph(runs, 20) for _ in range(3)]))
             del runs
             torch.cuda.empty_cache()
             var[name] = {"us": us, "TOP/s": ops / us / 1e6}
