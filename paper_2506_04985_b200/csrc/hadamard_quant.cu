@@ -115,16 +115,20 @@ __global__ void __launch_bounds__(256) hadamard_quant_kernel(const HadQuantParam
 constexpr int kTrStride = 68;                        // floats per transposed row: 16-byte stores of 8 lanes hit 8 bank groups
 constexpr int kTrWarp = 32 * kTrStride;              // floats per warp
 
-template <bool kSilu>
+// kTwo: groups of 4096 channels, two warps per group: each warp does the above for its half, then the
+// halves meet in the last stage (distance 2048) through the same tile -- warp 0 keeps a + b, warp 1 a - b.
+template <bool kSilu, bool kTwo = false>
 __global__ void __launch_bounds__(256, 3) hadamard2048_quant_kernel(const HadQuantParams P) {
   extern __shared__ __align__(16) float tr_all[];
   pdl_wait();                                    // the products come from the matmul before this kernel
   pdl_launch_dependents();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int groups = P.K >> 11;
-  const long long wid = (long long)blockIdx.x * 8 + warp;
-  if (wid >= (long long)P.M * groups) return;    // (warps never meet at a CTA-wide barrier)
-  const int t = (int)(wid / groups), grp = (int)(wid % groups);
+  const int groups = P.K >> (kTwo ? 12 : 11);
+  const int half = kTwo ? (warp & 1) : 0;        // which 2048 channels of a 4096-channel group
+  const long long wid = kTwo ? (long long)blockIdx.x * 4 + (warp >> 1) : (long long)blockIdx.x * 8 + warp;
+  if (wid >= (long long)P.M * groups) return;    // (both warps of a group leave together; no CTA-wide barrier)
+  const int t = (int)(wid / groups);
+  const int grp = (int)(wid % groups) * (kTwo ? 2 : 1) + half;     // in units of 2048 channels
   const uint4* row = P.X + (size_t)t * (size_t)(P.ldx >> 3);
   float* tr = tr_all + warp * kTrWarp;
   // The group's 256 chunks of 8 channels arrive in fully coalesced loads (lane l takes chunks
@@ -197,6 +201,22 @@ __global__ void __launch_bounds__(256, 3) hadamard2048_quant_kernel(const HadQua
         unpack_f32x2(add_f32x2(a, b), x[2 * l], x[2 * l + 1]);
         unpack_f32x2(sub_f32x2(a, b), x[2 * (l + d)], x[2 * (l + d) + 1]);
       }
+  if constexpr (kTwo) {
+    // distance 2048: channel c of the first half with channel c of the second.  Each warp parks its
+    // 64 values per lane in its own tile (word 32 j + lane), the pair meets at a named barrier, reads
+    // the partner's values, and meets again before the tiles are reused for the codes.
+    __syncwarp();                                // every lane has read the transposed tile
+#pragma unroll
+    for (int j = 0; j < 64; ++j) tr[32 * j + lane] = x[j];
+    named_bar_sync(1 + (warp >> 1), 64);
+    const float* other = tr_all + (warp ^ 1) * kTrWarp;
+#pragma unroll
+    for (int j = 0; j < 64; ++j) {
+      const float y = other[32 * j + lane];
+      x[j] = half ? __fsub_rn(y, x[j]) : __fadd_rn(x[j], y);
+    }
+    named_bar_sync(1 + (warp >> 1), 64);
+  }
   const float p = P.s_in ? __ldg(P.s_in + t) : 1.0f;
   const QuantConsts qc = quant_consts(p, P.inv_delta, P.qmax_minus_z, P.flip);
   __syncwarp();                                  // every lane has read the tile before it is overwritten
@@ -214,16 +234,20 @@ __global__ void __launch_bounds__(256, 3) hadamard2048_quant_kernel(const HadQua
   }
 }
 
-static cudaError_t launch_had2048(const HadQuantParams& P, cudaStream_t st) {
-  const long long warps = (long long)P.M * (P.K / 2048);
+template <bool kSilu, bool kTwo>
+static cudaError_t launch_had_tr(const HadQuantParams& P, cudaStream_t st) {
+  const long long warps = (long long)P.M * (P.K / 2048);          // 8 per CTA either way
   const size_t smem = (size_t)8 * kTrWarp * sizeof(float);
-  static PerDeviceInt attr_a, attr_b;
-  if (P.silu_inter) {
-    if (!ensure_smem_attr(attr_a, hadamard2048_quant_kernel<true>, (int)smem)) return cudaErrorInvalidValue;
-    return launch_kernel(hadamard2048_quant_kernel<true>, dim3((unsigned)((warps + 7) / 8)), dim3(256), smem, st, true, P);
-  }
-  if (!ensure_smem_attr(attr_b, hadamard2048_quant_kernel<false>, (int)smem)) return cudaErrorInvalidValue;
-  return launch_kernel(hadamard2048_quant_kernel<false>, dim3((unsigned)((warps + 7) / 8)), dim3(256), smem, st, true, P);
+  static PerDeviceInt attr;
+  if (!ensure_smem_attr(attr, hadamard2048_quant_kernel<kSilu, kTwo>, (int)smem)) return cudaErrorInvalidValue;
+  return launch_kernel(hadamard2048_quant_kernel<kSilu, kTwo>, dim3((unsigned)((warps + 7) / 8)), dim3(256), smem, st, true, P);
+}
+
+static cudaError_t launch_had2048(const HadQuantParams& P, cudaStream_t st) {
+  return P.silu_inter ? launch_had_tr<true, false>(P, st) : launch_had_tr<false, false>(P, st);
+}
+static cudaError_t launch_had4096(const HadQuantParams& P, cudaStream_t st) {
+  return P.silu_inter ? launch_had_tr<true, true>(P, st) : launch_had_tr<false, true>(P, st);
 }
 
 template <int C>
@@ -254,7 +278,7 @@ cudaError_t hadamard_quant_launch(cudaStream_t st, const void* X, int M, int K, 
     case 512: return launch_had<2>(P, st);
     case 1024: return launch_had<4>(P, st);
     case 2048: return launch_had2048(P, st);
-    case 4096: return launch_had<16>(P, st);
+    case 4096: return launch_had4096(P, st);
     default: return cudaErrorInvalidValue;
   }
 }

@@ -11,7 +11,7 @@ from helpers import dev, host, oqp, bf16_host, assert_bf16_close
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("M,K", [(5, 256), (33, 768), (64, 1024), (7, 3584), (9, 14336), (3, 28672), (130, 2048)])
+@pytest.mark.parametrize("M,K", [(5, 256), (33, 768), (64, 1024), (7, 3584), (9, 14336), (3, 28672), (37, 4096), (21, 12288), (130, 2048)])
 @pytest.mark.parametrize("sym", [True, False])
 def test_hadamard_quant_codes_bit_exact(M, K, sym):
     m = synth.activations(M, K, 6, f"had/m{K}", law="student_t3", outlier_frac=0.01, outlier_gain=30.0)
